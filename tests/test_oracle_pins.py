@@ -1,0 +1,329 @@
+"""Pins the CPU oracle to things other than itself: closed forms, library routines,
+hand-worked fixtures, brute force on tiny inputs and invariants.  No GPU needed."""
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import codecomp_oracle as orc
+from paper_2604_10235_b200 import inputs as gen
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rand(shape, seed):
+    return np.random.Generator(np.random.PCG64(seed)).standard_normal(shape)
+
+
+# ------------------------------------------------------------------ bf16 widening
+def test_bf16_widening_matches_torch():
+    bits = np.arange(0, 65536, 7, dtype=np.uint16)
+    bits = bits[(bits & 0x7F80) != 0x7F80]          # finite patterns only
+    ref = torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).double().numpy()
+    np.testing.assert_array_equal(orc.bf16_bits_to_f64(bits), ref)
+
+
+def test_generator_bf16_rounding_matches_torch():
+    x = _rand(4096, 3).astype(np.float32)
+    ref = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    np.testing.assert_array_equal(gen.f32_to_bf16_bits(x), ref)
+
+
+# ------------------------------------------------------------------ window scores
+def brute_scores(q, k, n_heads_kv):
+    """Triple-loop restatement of Section 4.5 with grouped heads, pure Python floats."""
+    w, hq, d = q.shape
+    n = k.shape[0]
+    g = hq // n_heads_kv
+    u = [[0.0] * n for _ in range(n_heads_kv)]
+    for head in range(hq):
+        h = head // g
+        for t in range(w):
+            s = [sum(float(q[t, head, c]) * float(k[j, h, c]) for c in range(d)) / math.sqrt(d)
+                 for j in range(n)]
+            z = sum(math.exp(x) for x in s)
+            for j in range(n):
+                u[h][j] += math.exp(s[j]) / z
+    return np.array(u)
+
+
+@pytest.mark.parametrize("w,hq,hkv,n,d", [(1, 1, 1, 5, 4), (3, 4, 2, 9, 8), (2, 6, 2, 17, 16),
+                                          (4, 3, 3, 7, 8)])
+def test_scores_vs_brute_force(w, hq, hkv, n, d):
+    q, k = _rand((w, hq, d), 11), _rand((n, hkv, d), 12)
+    u, _ = orc.window_scores(q, k, hkv)
+    np.testing.assert_allclose(u, brute_scores(q, k, hkv), rtol=1e-12, atol=1e-14)
+
+
+def test_single_row_is_library_softmax():
+    d, n = 128, 300
+    q, k = _rand((1, 1, d), 1), _rand((n, 1, d), 2)
+    u, lse = orc.window_scores(q, k, 1)
+    s = torch.from_numpy(k[:, 0, :] @ q[0, 0]) / math.sqrt(d)
+    np.testing.assert_allclose(u[0], torch.softmax(s, 0).numpy(), rtol=1e-12)
+    np.testing.assert_allclose(lse[0, 0], torch.logsumexp(s, 0).item(), rtol=1e-13)
+
+
+def test_two_key_closed_form_golden():
+    with open(os.path.join(GOLD, "two_key_softmax.json")) as f:
+        cases = json.load(f)["cases"]
+    for c in cases:
+        d = c["d"]
+        q = np.zeros((c["w"], 1, d)); q[:, 0, 0] = c["q"]
+        k = np.zeros((2, 1, d)); k[0, 0, 0] = c["a"]; k[1, 0, 0] = c["b"]
+        u, _ = orc.window_scores(q, k, 1)
+        np.testing.assert_allclose(u[0], c["u"], rtol=1e-13)
+
+
+def test_scores_invariants_and_special_cases():
+    w, hq, hkv, n, d = 5, 6, 2, 40, 32
+    q, k = _rand((w, hq, d), 5), _rand((n, hkv, d), 6)
+    u, _ = orc.window_scores(q, k, hkv)
+    g = hq // hkv
+    np.testing.assert_allclose(u.sum(axis=1), w * g, rtol=1e-12)        # rows of A sum to 1
+    # identical keys or a zero query -> uniform attention
+    u_c, _ = orc.window_scores(q, np.broadcast_to(k[:1], k.shape).copy(), hkv)
+    np.testing.assert_allclose(u_c, w * g / n, rtol=1e-12)
+    u_0, _ = orc.window_scores(np.zeros_like(q), k, hkv)
+    np.testing.assert_allclose(u_0, w * g / n, rtol=1e-12)
+    # adding one vector to every key shifts each softmax row by a constant
+    u_s, _ = orc.window_scores(q, k + _rand((1, hkv, d), 7), hkv)
+    np.testing.assert_allclose(u_s, u, rtol=1e-10)
+    # a key far in the query's direction takes all the mass of that head's rows
+    qpos = np.abs(q)
+    k3 = np.abs(k); k3[3, 0, :] = 1e3
+    u_p, _ = orc.window_scores(qpos, k3, hkv)
+    np.testing.assert_allclose(u_p[0, 3], w * g, rtol=1e-9)
+    # permuting the keys permutes the scores
+    perm = np.random.Generator(np.random.PCG64(9)).permutation(n)
+    u_perm, _ = orc.window_scores(q, k[perm], hkv)
+    np.testing.assert_allclose(u_perm, u[:, perm], rtol=1e-12)
+
+
+def test_gqa_head_mapping():
+    """Query head i belongs to KV head i // G: give KV head 1 identical keys (uniform
+    scores) and KV head 0 distinct ones."""
+    w, hq, hkv, n, d = 2, 4, 2, 12, 8
+    q, k = _rand((w, hq, d), 21), _rand((n, hkv, d), 22)
+    k[:, 1, :] = k[0, 1, :]
+    u, lse = orc.window_scores(q, k, hkv)
+    np.testing.assert_allclose(u[1], w * 2 / n, rtol=1e-12)
+    assert np.ptp(u[0]) > 1e-3
+    # lse of the uniform head: s + log n
+    s = (q[:, 2:, :] * k[0, 1, :]).sum(-1) / math.sqrt(d)            # [w][2]
+    np.testing.assert_allclose(lse[2:], (s + math.log(n)).T, rtol=1e-12)
+
+
+# ------------------------------------------------------------------ pooling
+@pytest.mark.parametrize("width", [1, 3, 5, 7])
+@pytest.mark.parametrize("n", [1, 2, 6, 50])
+def test_pool_matches_library(width, n):
+    u = np.abs(_rand((3, n), 30 + n))
+    t = torch.from_numpy(u)[None]
+    mx = torch.nn.functional.max_pool1d(t, width, 1, width // 2)[0].numpy()
+    av = torch.nn.functional.avg_pool1d(t, width, 1, width // 2, count_include_pad=True)[0].numpy()
+    np.testing.assert_array_equal(orc.pool_scores(u, orc.POOL_MAX, width), mx)
+    np.testing.assert_allclose(orc.pool_scores(u, orc.POOL_AVG, width), av, rtol=1e-13)
+    np.testing.assert_array_equal(orc.pool_scores(u, orc.POOL_NONE, width), u)
+
+
+def test_pool_closed_forms():
+    delta = np.zeros((1, 21)); delta[0, 10] = 2.0
+    mx = orc.pool_scores(delta, orc.POOL_MAX, 7)
+    assert mx[0].tolist() == [0.0] * 7 + [2.0] * 7 + [0.0] * 7          # plateau of width k
+    const = np.full((1, 9), 3.0)
+    av = orc.pool_scores(const, orc.POOL_AVG, 5)[0]
+    np.testing.assert_allclose(av, [3 * 3 / 5, 3 * 4 / 5, 3, 3, 3, 3, 3, 3 * 4 / 5, 3 * 3 / 5])
+    u32 = np.abs(_rand((2, 33), 31)).astype(np.float32)
+    out = orc.pool_scores(u32, orc.POOL_AVG, 5, dtype=np.float32)
+    assert out.dtype == np.float32
+    j = 7                                            # left-to-right fp32 sum, then divide
+    acc = np.float32(0)
+    for o in range(-2, 3):
+        acc = np.float32(acc + u32[1, j + o])
+    assert out[1, j] == np.float32(acc / np.float32(5))
+
+
+# ------------------------------------------------------------------ fuse
+def test_fuse_hand_values():
+    out = orc.fuse_prior(np.array([[2.0, 4.0]]), np.array([1.0, 0.5]), 0.25, 3.0)
+    assert out.tolist() == [[3.5, 2.5]]
+    a, b = np.float32(0.1), np.float32(0.7)
+    x, p = np.float32(1.2345678), np.float32(0.3333333)
+    out32 = orc.fuse_prior(np.array([[x]], np.float32), np.array([p], np.float32), 0.1, 0.7,
+                           dtype=np.float32)
+    assert out32.dtype == np.float32 and out32[0, 0] == np.float32(np.float32(a * x) + np.float32(b * p))
+
+
+# ------------------------------------------------------------------ selection
+def brute_select(fused, prior, lens, budget, theta, span_ratio, span_min):
+    """Rank every item by counting the items that precede it (O(m^2)), then walk ranks."""
+    m = len(fused)
+    forced = [np.float32(prior[i]) >= np.float32(theta) for i in range(m)]
+    if span_ratio > 0:
+        cap = min(budget, max(span_min, math.floor(span_ratio * budget + 1e-9)))
+        cand = [i for i in range(m) if forced[i]]
+
+        def before_p(a, b):
+            return prior[a] > prior[b] or (prior[a] == prior[b] and a < b)
+        ranked = sorted(cand, key=lambda i: sum(before_p(o, i) for o in cand))
+        forced = [False] * m
+        tot = 0
+        for i in ranked:
+            tot += lens[i]
+            if tot > cap:
+                break
+            forced[i] = True
+
+    def before(a, b):
+        if forced[a] != forced[b]:
+            return forced[a]
+        if forced[a]:
+            return a < b                      # protected tokens: sequence order only
+        if fused[a] != fused[b]:
+            return fused[a] > fused[b]
+        return a < b
+    rank = [sum(before(o, i) for o in range(m) if o != i) for i in range(m)]
+    by_rank = sorted(range(m), key=lambda i: rank[i])
+    take = [0] * m
+    left = min(budget, sum(lens))
+    for i in by_rank:
+        take[i] = min(lens[i], left)
+        left -= take[i]
+    return np.array(take)
+
+
+def test_select_golden_cases():
+    with open(os.path.join(GOLD, "select_cases.json")) as f:
+        cases = json.load(f)["cases"]
+    for c in cases:
+        n = c.get("n", len(c["fused"]))
+        idx = orc.select_tokens(np.array(c["fused"]), np.array(c["prior"], np.float32), n,
+                                c["budget"], c["theta"], c["span_ratio"], c["span_min"],
+                                c["chunk"])
+        assert idx.tolist() == c["idx"], c["name"]
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_select_vs_brute_force(seed):
+    rng = np.random.Generator(np.random.PCG64(100 + seed))
+    m = int(rng.integers(1, 40))
+    chunk = int(rng.choice([1, 1, 3, 4]))
+    n = m * chunk - int(rng.integers(0, chunk))
+    lens = orc.chunk_lengths(n, chunk)
+    m = len(lens)
+    fused = rng.choice(np.round(rng.random(6), 2), size=m)            # many exact ties
+    prior = rng.choice([0.0, 0.0, 0.3, 0.6, 0.9], size=m).astype(np.float32)
+    budget = int(rng.integers(0, n + 3))
+    ratio = float(rng.choice([0.0, 0.5, 0.7]))
+    take = orc.select_items(fused, prior, lens, budget, 0.5, ratio, 2)
+    ref = brute_select(fused, prior, lens, budget, 0.5, ratio, 2)
+    np.testing.assert_array_equal(take, ref)
+
+
+def test_select_invariants():
+    rng = np.random.Generator(np.random.PCG64(77))
+    n = 500
+    fused = rng.random(n)
+    prior = (rng.random(n) < 0.1).astype(np.float32)
+    forced = np.flatnonzero(prior >= 0.5)
+    for budget in [0, 1, len(forced) - 1, len(forced), len(forced) + 10, n - 1, n, n + 5]:
+        idx = orc.select_tokens(fused, prior, n, budget, 0.5)
+        assert len(idx) == min(budget, n)                               # count = B exactly
+        assert np.all(np.diff(idx) > 0)                                 # ascending, unique
+        if budget >= len(forced):
+            assert set(forced) <= set(idx.tolist())                     # all protected kept
+            rest = np.setdiff1d(idx, forced)
+            out = np.setdiff1d(np.arange(n), idx)
+            if len(rest) and len(out):
+                assert fused[rest].min() >= fused[out].max()
+        else:
+            assert idx.tolist() == forced[:budget].tolist()             # first B of P
+
+
+def test_span_budget_hand_values():
+    assert orc.span_budget(100, 0.5, 16) == 50
+    assert orc.span_budget(20, 0.5, 16) == 16
+    assert orc.span_budget(10, 0.5, 16) == 10
+    assert orc.span_budget(10, 0.7, 0) == 7
+    assert orc.span_budget(100, 0.29, 0) == 29
+
+
+# ------------------------------------------------------------------ chunks
+def test_chunk_reduce_definition():
+    u = _rand((2, 23), 40)
+    p = np.zeros(23, np.float32); p[[4, 22]] = [0.7, 0.2]
+    us, ps = orc.chunk_reduce(u, p, 10)
+    for c, (lo, hi) in enumerate([(0, 10), (10, 20), (20, 23)]):
+        acc = u[:, lo].copy()
+        for j in range(lo + 1, hi):
+            acc = acc + u[:, j]
+        np.testing.assert_array_equal(us[:, c], acc)
+    assert ps.tolist() == [np.float32(0.7), 0.0, np.float32(0.2)]
+    np.testing.assert_allclose(us.sum(1), u.sum(1), rtol=1e-12)
+    assert orc.chunk_lengths(23, 10).tolist() == [10, 10, 3]
+    assert orc.chunk_lengths(20, 10).tolist() == [10, 10]
+
+
+# ------------------------------------------------------------------ compaction / paged layout
+def test_compact_is_row_gather():
+    k = np.arange(6 * 2 * 4, dtype=np.uint16).reshape(6, 2, 4)
+    v = k + 1000
+    idx = [np.array([0, 5]), np.array([2, 3, 4])]
+    ko, vo = orc.compact_kv(k, v, idx)
+    for h in range(2):
+        for s, j in enumerate(idx[h]):
+            assert ko[h][s].tolist() == k[j, h].tolist()
+            assert vo[h][s].tolist() == v[j, h].tolist()
+
+
+def test_paged_helpers():
+    table = np.array([7, 2, 9], dtype=np.int32)
+    rows = orc.paged_rows(table, 10, 4)
+    assert rows.tolist() == [28, 29, 30, 31, 8, 9, 10, 11, 36, 37]
+    pages = orc.assign_output_pages([5, 0, 9], [100, 100, 6], 4, np.arange(50, 60))
+    assert [p.tolist() for p in pages] == [[50, 51], [], [52, 53]]
+
+
+# ------------------------------------------------------------------ whole path
+def test_compress_sequence_invariants_on_tiny_workload():
+    wl = gen.workloads()["tiny"]
+    x = gen.make_layer(wl)
+    res = orc.compress_sequence(x.q_win[0], x.k, x.v, x.prior, wl.n_heads_kv, wl.pool_kind,
+                                wl.pool_size, wl.budget, wl.alpha, wl.beta, wl.force_threshold)
+    g = wl.group
+    np.testing.assert_allclose(res["scores"].sum(1), wl.window * g, rtol=1e-12)
+    forced = np.flatnonzero(x.prior >= 0.5)
+    assert 0 < len(forced) < wl.budget
+    for h in range(wl.n_heads_kv):
+        idx = res["idx"][h]
+        assert len(idx) == wl.budget and np.all(np.diff(idx) > 0)
+        assert set(forced) <= set(idx.tolist())
+        np.testing.assert_array_equal(res["k_out"][h], x.k[idx, h])
+        np.testing.assert_array_equal(res["v_out"][h], x.v[idx, h])
+        assert np.all(res["pooled"][h] >= res["scores"][h])             # max-pool dominates
+
+
+def test_workload_recipe_statistics():
+    wls = gen.workloads()
+    p, lab = gen.structural_prior(1, 200000)
+    assert abs(p.mean() - 0.0666) < 0.004                 # 0.29 * E[min(3, len)] / 12
+    assert set(np.unique(p)) == {0.0, 1.0}
+    assert wls["ragged_paged"].lens == gen.workloads()["ragged_paged"].lens   # seeded
+    assert all(8192 <= s <= 65536 for s in wls["ragged_paged"].lens)
+    for dens, target in [("5", 0.05), ("15", 0.15), ("30", 0.30)]:
+        v = gen.qwen_variant(wls["qwen25_coder_7b"], 4096, dens)
+        pp, _ = gen.structural_prior(2, 200000, v.p_structural, v.flagged_per_line)
+        assert abs(pp.mean() - target) < 0.012
+    small = gen.Workload("s", 9, 1, 4, 2, 128, 8, gen.POOL_MAX, 3, 8, seq_lens=(40, 70),
+                         budget_frac=0.1, page_size=16)
+    x = gen.make_layer(small)
+    assert x.page_table.shape == (2, 5) and x.k.shape[0] == x.pool_pages * 16
+    y = gen.make_layer(gen.Workload("s", 9, 1, 4, 2, 128, 8, gen.POOL_MAX, 3, 8, seq_lens=(40, 70),
+                                    budget_frac=0.1))
+    rows = orc.paged_rows(x.page_table[1], 70, 16)
+    np.testing.assert_array_equal(x.k[rows], y.k[40:110])                  # same bits, scattered
+    assert len(set(x.free_pages.tolist()) & set(x.page_table[x.page_table >= 0].tolist())) == 0
