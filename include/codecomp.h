@@ -1,0 +1,178 @@
+/*
+ * codecomp.h - C ABI of the CodeComp per-layer KV-cache compression step on one B200.
+ *
+ * The step runs once per transformer layer after prefill (paper, Section 4.5:
+ * "Compression is applied independently at each transformer layer"):
+ *
+ *   score   u_h(j) = sum over the window rows t and the query heads g of KV head h of
+ *           softmax_j( q_{g,t} . k_j / sqrt(d) )                       (Section 4.5)
+ *   pool    1-D sliding-window pooling of u along the token axis   (Appendix, "Compression settings")
+ *   fuse    f(j) = alpha * pooled(j) + beta * prior(j); tokens whose structural prior
+ *           reaches a threshold are protected                 (Section 4.4, "Span scoring",
+ *                                                              "Token-level protection")
+ *   select  protected tokens first, then the top-ranked f, until the budget B is full
+ *                                                              (Sections 4.4 and 4.5)
+ *   compact gather the retained K/V rows, in original order, into a new cache
+ *                                                              (Section 4.6: positions are kept)
+ *
+ * Conventions
+ *  - Every function returns CC_OK (0) or a negative CC_ERR_* code; cc_last_error() gives a
+ *    text for the last failure of a context.  Nothing is thrown, nothing aborts.
+ *  - "device" pointers are CUDA device memory of the context's GPU, "host" pointers are
+ *    ordinary memory.  The caller owns every buffer.  The library allocates nothing per
+ *    call, never synchronises the device, and only enqueues work on the given stream
+ *    (a cudaStream_t passed as void*; NULL is the default stream).  Results are valid
+ *    once that stream has reached the end of the enqueued work.
+ *  - A cc_layer_desc is host memory and is read during the call only.
+ *  - bf16 tensors have head_dim contiguous; the other strides are given in elements.
+ *  - One cc_ctx must not be used from two threads at once.
+ *
+ * Layout of a batch.  num_seqs == 0 means one sequence of `n` tokens and budget `budget`.
+ * num_seqs >= 1 (at most CC_MAX_SEQS) means a ragged batch described by the host arrays
+ * seq_lens / budgets.  With tok_off[s] = sum of earlier n_s, item_off[s] = sum of earlier
+ * ceil(n_s / chunk) and idx_off[s] = sum of earlier budgets B_s:
+ *    q_win   bf16 [S][w][H_q][d]          strides q_stride_seq / q_stride_row / q_stride_head
+ *    k, v    bf16 page_size == 0: token j of sequence s is row tok_off[s] + j of
+ *                 [N_tot][H_kv][d] (strides kv_stride_tok / kv_stride_head);
+ *                 page_size > 0: it is row page_table[s][j / page_size] * page_size +
+ *                 j % page_size of the same kind of array (the page pool)
+ *    prior   f32  [N_tot]                 sequence s at tok_off[s]
+ *    scores  f32  [H_kv][N_tot]           sequence s at column tok_off[s]
+ *    lse     f32  [S][H_q][w]             natural-log sum of exp of the scaled logits
+ *    fused   f32  [H_kv][M_tot]           one value per item (token, or chunk if chunk_size > 1)
+ *    idx     i32  [H_kv][B_tot]           sequence s at column idx_off[s]; token indices within
+ *                                         the sequence, ascending; entries past count are -1
+ *    count   i32  [S][H_kv]               min(B_s, n_s)
+ *    k_out, v_out  page_size == 0: slot i of sequence s is row idx_off[s] + i of
+ *                 [B_tot][H_kv][d] (strides out_stride_tok / out_stride_head, 0 = dense);
+ *                 page_size > 0: it is row out_page_table[s][i / page_size] * page_size +
+ *                 i % page_size of the pool given as k_out / v_out (same strides as k, v).
+ */
+#ifndef CODECOMP_H_
+#define CODECOMP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CC_OK                0
+#define CC_ERR_INVALID_ARG  (-1)  /* NULL pointer, negative size, inconsistent descriptor */
+#define CC_ERR_UNSUPPORTED  (-2)  /* head_dim != 128, w*G > 512, even pool width, wrong GPU ... */
+#define CC_ERR_WORKSPACE    (-3)  /* workspace NULL, misaligned or smaller than cc_workspace_bytes */
+#define CC_ERR_CUDA         (-4)  /* a CUDA runtime/driver call failed; see cc_last_error */
+#define CC_ERR_TIMEOUT      (-5)  /* device status only: a bounded wait inside a kernel ran out */
+#define CC_ERR_DEVICE_FLAG  (-6)  /* device status only: a kernel met an invalid page id or index */
+
+#define CC_BF16        1
+#define CC_MODE_BF16   0   /* tensor-core scores: bf16 operands, fp32 accumulate and softmax */
+#define CC_MODE_FP32   1   /* verification mode: every product and sum in fp32 on CUDA cores */
+#define CC_POOL_NONE   0
+#define CC_POOL_MAX    1
+#define CC_POOL_AVG    2
+#define CC_MAX_SEQS    64
+
+typedef struct cc_ctx cc_ctx;
+
+typedef struct cc_layer_desc {
+  int32_t n_heads_q;        /* H_q, a multiple of n_heads_kv */
+  int32_t n_heads_kv;       /* H_kv */
+  int32_t head_dim;         /* d, must be 128 */
+  int32_t window;           /* w: rows of the observation window (Section 4.5, W) */
+  int32_t dtype;            /* CC_BF16 */
+  int32_t compute_mode;     /* CC_MODE_BF16 or CC_MODE_FP32 */
+  int32_t pool_kind;        /* CC_POOL_* */
+  int32_t pool_size;        /* odd width k <= 63, centred, stride 1 */
+  int32_t chunk_size;       /* <= 1: token level; c > 1: rank fixed chunks of c tokens (no pooling) */
+  float   alpha, beta;      /* f = alpha * pooled + beta * prior */
+  float   force_threshold;  /* prior >= threshold => protected; +INFINITY disables protection */
+  double  span_ratio;       /* rho_span; <= 0: no cap on protected tokens.  > 0: protected tokens
+                               are limited to B_span = min(B, max(span_min, floor(rho * B))),
+                               taken by (prior descending, index ascending)  (Section 4.4) */
+  int32_t span_min;         /* B_min */
+  int32_t n;                /* single sequence: prefix length (L_c in Section 4.5) */
+  int32_t budget;           /* single sequence: B, tokens kept per KV head */
+  int64_t q_stride_seq, q_stride_row, q_stride_head;   /* elements */
+  int64_t kv_stride_tok, kv_stride_head;               /* elements */
+  int64_t out_stride_tok, out_stride_head;             /* elements; 0 = dense [.][H_kv][d] */
+  int32_t num_seqs;         /* 0 = single sequence */
+  int32_t page_size;        /* 0 = contiguous; else 8, 16, 32, 64 or 128 tokens per page */
+  const int32_t* seq_lens;  /* HOST [num_seqs] */
+  const int32_t* budgets;   /* HOST [num_seqs] */
+  const int32_t* page_table;/* DEVICE [num_seqs][page_table_stride], used when page_size > 0 */
+  int32_t page_table_stride;
+  int32_t out_page_table_stride; /* row length of out_page_table (>= ceil(B_s / page_size)) */
+} cc_layer_desc;
+
+/* Creates a context on CUDA device `device` (must be compute capability 10.x).  Allocates a
+ * few hundred bytes of device and pinned host memory for the status word; the only
+ * allocation the library ever makes.  *out is untouched on failure. */
+int cc_create(cc_ctx** out, int device);
+/* Frees the context.  The caller must have synchronised every stream that used it. */
+int cc_destroy(cc_ctx* ctx);
+/* Static text for a status code. */
+const char* cc_status_string(int status);
+/* Text describing the last failure recorded on `ctx` (empty string if none). */
+const char* cc_last_error(const cc_ctx* ctx);
+/* Synchronises `stream`, then reports and clears the device-side status word: CC_OK, or
+ * CC_ERR_TIMEOUT / CC_ERR_DEVICE_FLAG if a kernel gave up a bounded wait or skipped an
+ * invalid page id.  Outputs of a call that reported an error are unspecified. */
+int cc_poll_status(cc_ctx* ctx, void* stream, int* device_status);
+
+/* Bytes of device workspace (256-byte aligned) that any entry point below needs for `desc`.
+ * Returns 0 if the descriptor is invalid. */
+size_t cc_workspace_bytes(const cc_ctx* ctx, const cc_layer_desc* desc);
+
+/* A1 - window attention scores (Section 4.5, the equation for A and u(j)), summed over the
+ * query heads of each KV head.  q_win, k: device bf16.  scores: device f32 [H_kv][N_tot],
+ * fully overwritten.  lse: device f32 [S][H_q][w] or NULL.  ws: device workspace. */
+int cc_score_window(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win, const void* k,
+                    float* scores, float* lse, void* ws, size_t ws_bytes, void* stream);
+
+/* A2+A3 - pooling (Appendix "Compression settings") and prior fusion (Section 4.4 "Span
+ * scoring").  Token level: fused[h][j] = alpha * pool(scores[h])[j] + beta * prior[j], every
+ * operation rounded to f32, average pooling = left-to-right sum of the k zero-padded taps
+ * divided by k, max pooling over the valid taps.  Chunk level (chunk_size > 1): the item
+ * value is the in-order f32 sum of the chunk's scores and the prior is the chunk's maximum.
+ * scores, prior, fused: device f32.  Needs no workspace. */
+int cc_fuse_prior_pool(cc_ctx* ctx, const cc_layer_desc* desc, const float* scores,
+                       const float* prior, float* fused, void* stream);
+
+/* A4 - selection under the budget (Section 4.4 "Token-level protection", "Span selection
+ * under budget"; Section 4.5).  Items are ranked: protected first (in sequence order), then
+ * larger fused value, then lower index; items are taken in rank order until min(B_s, n_s)
+ * tokens are kept (a chunk that crosses the budget keeps its first tokens).  idx receives the
+ * retained token indices of each head in ascending order, -1 beyond count; count receives
+ * min(B_s, n_s).  fused: device f32 [H_kv][M_tot]; prior: device f32 [N_tot]. */
+int cc_topk_select(cc_ctx* ctx, const cc_layer_desc* desc, const float* fused,
+                   const float* prior, int32_t* idx, int32_t* count,
+                   void* ws, size_t ws_bytes, void* stream);
+
+/* A5 - compaction: k_out[slot i of head h] = k[token idx[h][i] of head h], same for v, as
+ * bit copies.  Paged layout: sequence s receives ceil(min(B_s, n_s) / page_size) page ids,
+ * taken in order from free_pages (device i32, sequences served in order), written to
+ * out_page_table[s][.] (device i32, -1 padded).  k_out/v_out must not alias k/v rows that
+ * are still to be read; in-place compaction is rejected when the pointers are equal and
+ * the layout is contiguous. */
+int cc_compact_kv(cc_ctx* ctx, const cc_layer_desc* desc, const void* k, const void* v,
+                  const int32_t* idx, void* k_out, void* v_out,
+                  const int32_t* free_pages, int32_t* out_page_table, void* stream);
+
+/* A8 - the whole step: score, pool, fuse, select, compact, enqueued back to back with the
+ * intermediates (scores, fused values) in the workspace and no host synchronisation. */
+int cc_compress_layer(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win, const void* k,
+                      const void* v, const float* prior, void* k_out, void* v_out,
+                      int32_t* idx, int32_t* count, const int32_t* free_pages,
+                      int32_t* out_page_table, void* ws, size_t ws_bytes, void* stream);
+
+/* Device pointers, inside the workspace last given to cc_compress_layer for `desc`, of the
+ * intermediate scores [H_kv][N_tot] and fused values [H_kv][M_tot] (for inspection). */
+int cc_workspace_views(const cc_ctx* ctx, const cc_layer_desc* desc, void* ws,
+                       float** scores, float** fused);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* CODECOMP_H_ */

@@ -1,0 +1,102 @@
+// Internal declarations shared by the kernels and the C-ABI layer of libcodecomp.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <stdint.h>
+
+#include "codecomp.h"
+
+namespace cc {
+
+constexpr int kHeadDim = 128;
+constexpr int kTileKeys = 128;       // keys per score tile (tensor-core path)
+constexpr int kMaxRows = 512;        // w * G limit
+
+// Per-sequence geometry, derived on the host from the descriptor.
+struct SeqInfo {
+  int n;             // tokens
+  int budget;        // B_s as given
+  int keep;          // min(B_s, n)
+  int n_items;       // tokens, or chunks when chunk > 1
+  int tok_off;       // offset of the sequence in [N_tot] arrays
+  int item_off;      // offset in [M_tot] arrays
+  int idx_off;       // offset in [B_tot] arrays
+  int tile_off;      // first score tile of the sequence (per KV head)
+  int n_tiles;       // ceil(n / kTileKeys)
+  int out_page_off;  // first entry of free_pages used by the sequence
+  int span_cap;      // B_span, or -1 when protected tokens are not capped
+  int pad_;
+};
+
+struct BatchTable {
+  int num_seqs;
+  int page_size;     // 0 = contiguous
+  int chunk;         // >= 1
+  int n_tot, m_tot, b_tot;
+  int tiles_per_head;   // sum of n_tiles
+  int max_items;
+  SeqInfo seq[CC_MAX_SEQS];
+};
+
+struct Geometry {
+  int hq, hkv, group, window, rows;       // rows = window * group
+  int64_t q_stride_seq, q_stride_row, q_stride_head;
+  int64_t kv_stride_tok, kv_stride_head;
+  int64_t out_stride_tok, out_stride_head;
+  const int32_t* page_table;
+  int page_table_stride, out_page_table_stride;
+};
+
+// Device status word: [0] = first error code, [1] = detail (where it happened).
+struct DeviceStatus {
+  int code;
+  int detail;
+  int pad[2];
+};
+
+__device__ __forceinline__ void report_error(DeviceStatus* st, int code, int detail) {
+  if (atomicCAS(&st->code, 0, code) == 0) st->detail = detail;
+}
+
+// Pool row of token j of a sequence (paged or contiguous).  Returns -1 for a bad page id.
+__device__ __forceinline__ int64_t token_row(const BatchTable& bt, const Geometry& g, int s, int j,
+                                             int64_t pool_rows) {
+  if (bt.page_size == 0) return (int64_t)bt.seq[s].tok_off + j;
+  int page = g.page_table[(int64_t)s * g.page_table_stride + j / bt.page_size];
+  int64_t row = (int64_t)page * bt.page_size + j % bt.page_size;
+  if (page < 0 || (pool_rows > 0 && row >= pool_rows)) return -1;
+  return row;
+}
+
+struct Launch {
+  cudaStream_t stream;
+  DeviceStatus* status;
+  int sm_count;
+};
+
+// ---- kernels' host-side launchers (each returns a cudaError_t from the launch) ----------
+size_t score_simt_ws_bytes(const BatchTable& bt, const Geometry& g, int sm_count);
+cudaError_t launch_score_simt(const Launch& L, const BatchTable& bt, const Geometry& g,
+                              const void* q, const void* k, float* scores, float* lse, void* ws);
+
+size_t score_tc_ws_bytes(const BatchTable& bt, const Geometry& g, int sm_count);
+// encode = cuTensorMapEncodeTiled entry point; err receives a CUresult-like code on failure
+cudaError_t launch_score_tc(const Launch& L, const BatchTable& bt, const Geometry& g,
+                            const void* q, const void* k, float* scores, float* lse, void* ws,
+                            void* encode_fn, int64_t pool_rows, int* drv_err);
+
+cudaError_t launch_fuse_pool(const Launch& L, const BatchTable& bt, const Geometry& g,
+                             int pool_kind, int pool_size, float alpha, float beta,
+                             const float* scores, const float* prior, float* fused);
+
+size_t select_ws_bytes(const BatchTable& bt, const Geometry& g);
+cudaError_t launch_select(const Launch& L, const BatchTable& bt, const Geometry& g,
+                          float force_threshold, const float* fused, const float* prior,
+                          int32_t* idx, int32_t* count, void* ws);
+
+cudaError_t launch_compact(const Launch& L, const BatchTable& bt, const Geometry& g,
+                           const void* k, const void* v, const int32_t* idx, void* k_out,
+                           void* v_out, const int32_t* free_pages, int32_t* out_page_table);
+
+}  // namespace cc

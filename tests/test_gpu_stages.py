@@ -1,0 +1,269 @@
+"""Stage-by-stage parity of the CUDA path against the oracle, through the C ABI.
+Integer and byte outputs are compared bit for bit on identical fp32 inputs."""
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import codecomp_oracle as orc
+from paper_2604_10235_b200 import binding as cc
+from paper_2604_10235_b200 import inputs as gen
+
+from gpu_util import bf16_dev, bits_host, ctx, desc_for, f32_dev
+
+pytestmark = pytest.mark.gpu
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+GUARD = 64
+
+
+def guarded(shape, dtype, fill):
+    """Output tensor with guard words on both sides; returns (view, full, fill)."""
+    n = int(np.prod(shape))
+    full = torch.full((n + 2 * GUARD,), fill, dtype=dtype, device="cuda")
+    return full[GUARD:GUARD + n].view(*shape), full
+
+
+def guards_intact(full, fill):
+    return bool((full[:GUARD] == fill).all() and (full[-GUARD:] == fill).all())
+
+
+# ------------------------------------------------------------------ A2 + A3
+@pytest.mark.parametrize("n", [1, 2, 15, 129, 2048, 4099])
+@pytest.mark.parametrize("kind,width", [(cc.CC_POOL_NONE, 1), (cc.CC_POOL_MAX, 7), (cc.CC_POOL_MAX, 3),
+                                        (cc.CC_POOL_AVG, 5), (cc.CC_POOL_AVG, 1), (cc.CC_POOL_MAX, 63)])
+def test_fuse_prior_pool_token_level(n, kind, width):
+    rng = np.random.Generator(np.random.PCG64(n * 100 + width))
+    hkv = 3
+    u = np.abs(rng.standard_normal((hkv, n))).astype(np.float32) * np.float32(1e-3)
+    prior = (rng.random(n) < 0.2).astype(np.float32) * rng.random(n).astype(np.float32)
+    alpha, beta = 0.37, 1.25
+    d = cc.Desc(hkv * 2, hkv, 4, n=n, budget=1, pool_kind=kind, pool_size=width, alpha=alpha, beta=beta)
+    out, full = guarded((hkv, n), torch.float32, -7.0)
+    cc.cc_fuse_prior_pool(ctx(), d, f32_dev(u), f32_dev(prior), out)
+    ref = orc.fuse_prior(orc.pool_scores(u, kind, width, dtype=np.float32), prior[None, :], alpha,
+                         beta, dtype=np.float32)
+    np.testing.assert_array_equal(out.cpu().numpy(), ref)
+    assert guards_intact(full, -7.0)
+
+
+@pytest.mark.parametrize("n,chunk", [(23, 10), (20, 10), (5, 10), (32768, 10), (1000, 3)])
+def test_fuse_prior_pool_chunk_level(n, chunk):
+    rng = np.random.Generator(np.random.PCG64(n + chunk))
+    hkv = 2
+    u = np.abs(rng.standard_normal((hkv, n))).astype(np.float32)
+    prior = (rng.random(n) < 0.1).astype(np.float32)
+    d = cc.Desc(hkv, hkv, 4, n=n, budget=1, pool_kind=cc.CC_POOL_NONE, pool_size=1,
+                chunk_size=chunk, alpha=0.5, beta=2.0)
+    m = d.m_tot
+    out, full = guarded((hkv, m), torch.float32, -7.0)
+    cc.cc_fuse_prior_pool(ctx(), d, f32_dev(u), f32_dev(prior), out)
+    cu, cp = orc.chunk_reduce(u, prior, chunk, dtype=np.float32)
+    ref = orc.fuse_prior(cu, cp[None, :], 0.5, 2.0, dtype=np.float32)
+    np.testing.assert_array_equal(out.cpu().numpy(), ref)
+    assert guards_intact(full, -7.0)
+
+
+# ------------------------------------------------------------------ A4
+def run_select(fused, prior, n, budget, theta, span_ratio=0.0, span_min=0, chunk=1):
+    hkv = fused.shape[0]
+    d = cc.Desc(hkv, hkv, 4, n=n, budget=budget, pool_kind=cc.CC_POOL_NONE, pool_size=1,
+                chunk_size=chunk, force_threshold=theta, span_ratio=span_ratio, span_min=span_min)
+    idx_c, full = guarded((hkv, budget), torch.int32, -99)
+    count = torch.full((hkv,), -5, dtype=torch.int32, device="cuda")
+    cc.cc_topk_select(ctx(), d, f32_dev(fused), f32_dev(prior), idx_c, count)
+    assert ctx().poll() == 0
+    assert guards_intact(full, -99)
+    return idx_c.cpu().numpy(), count.cpu().numpy()
+
+
+def test_select_golden_cases():
+    with open(os.path.join(GOLD, "select_cases.json")) as f:
+        cases = json.load(f)["cases"]
+    for c in cases:
+        n = c.get("n", len(c["fused"]))
+        fused = np.array([c["fused"]], dtype=np.float32)
+        idx, count = run_select(fused, np.array(_token_prior(c, n), np.float32), n, c["budget"],
+                                c["theta"], c["span_ratio"], c["span_min"], c["chunk"])
+        keep = min(c["budget"], n)
+        assert count[0] == keep, c["name"]
+        assert idx[0, :keep].tolist() == c["idx"], c["name"]
+        assert (idx[0, keep:] == -1).all()
+
+
+def _token_prior(c, n):
+    """The fixtures give one prior per item; put it on the first token of each chunk."""
+    if c["chunk"] == 1:
+        return c["prior"]
+    p = [0.0] * n
+    for i, v in enumerate(c["prior"]):
+        p[i * c["chunk"]] = v
+    return p
+
+
+@pytest.mark.parametrize("n", [1, 15, 16, 17, 127, 128, 129, 2048, 4099, 32768, 65536])
+def test_select_matches_oracle_bit_exact(n):
+    rng = np.random.Generator(np.random.PCG64(n))
+    hkv = 2
+    u = (np.abs(rng.standard_normal((hkv, n))) * 1e-3).astype(np.float32)
+    fused = orc.pool_scores(u, orc.POOL_MAX, 7, dtype=np.float32)      # runs of exact ties
+    prior = (rng.random(n) < 0.07).astype(np.float32)
+    n_forced = int(prior.sum())
+    for budget in sorted({0, 1, n // 16, max(0, n_forced - 1), n_forced, n_forced + 3, n - 1, n, n + 5}):
+        if budget < 0:
+            continue
+        idx, count = run_select(fused, prior, n, budget, 0.5)
+        keep = min(budget, n)
+        for h in range(hkv):
+            ref = orc.select_tokens(fused[h], prior, n, budget, 0.5)
+            assert count[h] == keep
+            np.testing.assert_array_equal(idx[h, :keep], ref, err_msg=f"n={n} B={budget} h={h}")
+            assert (idx[h, keep:] == -1).all()
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_select_with_span_cap_and_graded_prior(seed):
+    rng = np.random.Generator(np.random.PCG64(500 + seed))
+    n = int(rng.integers(200, 5000))
+    hkv = 2
+    fused = rng.choice(rng.random(50).astype(np.float32), size=(hkv, n)).astype(np.float32)
+    prior = rng.choice(np.array([0, 0, 0, 0, 0.2, 0.6, 0.6, 0.8, 0.95], np.float32), size=n)
+    for budget in [n // 10, n // 3]:
+        for ratio, smin in [(0.5, 16), (0.25, 0), (1.0, 0)]:
+            idx, count = run_select(fused, prior, n, budget, 0.5, ratio, smin)
+            for h in range(hkv):
+                ref = orc.select_tokens(fused[h], prior, n, budget, 0.5, ratio, smin)
+                np.testing.assert_array_equal(idx[h, :len(ref)], ref)
+
+
+@pytest.mark.parametrize("n,chunk,budget", [(32768, 10, 2048), (1003, 10, 100), (95, 10, 95),
+                                            (4099, 7, 500), (64, 10, 7)])
+def test_select_chunk_level(n, chunk, budget):
+    rng = np.random.Generator(np.random.PCG64(n + budget))
+    hkv = 2
+    u = np.abs(rng.standard_normal((hkv, n))).astype(np.float32)
+    prior = (rng.random(n) < 0.02).astype(np.float32)
+    cu, cp = orc.chunk_reduce(u, prior, chunk, dtype=np.float32)
+    idx, count = run_select(cu, prior, n, budget, 0.5, chunk=chunk)
+    for h in range(hkv):
+        ref = orc.select_tokens(cu[h], cp, n, budget, 0.5, chunk=chunk)
+        np.testing.assert_array_equal(idx[h, :len(ref)], ref)
+        assert count[h] == len(ref) == min(budget, n)
+
+
+def test_select_negative_and_zero_scores():
+    n = 300
+    rng = np.random.Generator(np.random.PCG64(3))
+    fused = rng.standard_normal((1, n)).astype(np.float32)
+    fused[0, ::5] = 0.0
+    fused[0, 1::7] = -0.0
+    prior = np.zeros(n, np.float32)
+    for budget in [10, 150, 290]:
+        idx, _ = run_select(fused, prior, n, budget, 0.5)
+        np.testing.assert_array_equal(idx[0], orc.select_tokens(fused[0], prior, n, budget, 0.5))
+
+
+# ------------------------------------------------------------------ A5
+@pytest.mark.parametrize("n,budget,hkv", [(1, 1, 1), (129, 40, 2), (4099, 4099, 8), (2048, 512, 2)])
+def test_compact_contiguous(n, budget, hkv):
+    rng = np.random.Generator(np.random.PCG64(n + budget))
+    k = rng.integers(0, 65535, size=(n, hkv, 128), dtype=np.uint16)
+    v = rng.integers(0, 65535, size=(n, hkv, 128), dtype=np.uint16)
+    idx = np.stack([np.sort(rng.choice(n, size=budget, replace=False)) for _ in range(hkv)]).astype(np.int32)
+    d = cc.Desc(hkv, hkv, 4, n=n, budget=budget)
+    ko, kfull = guarded((budget, hkv, 128), torch.int16, 0x1111)
+    vo, vfull = guarded((budget, hkv, 128), torch.int16, 0x1111)
+    cc.cc_compact_kv(ctx(), d, bf16_dev(k), bf16_dev(v), torch.from_numpy(idx).cuda(),
+                     ko.view(torch.bfloat16), vo.view(torch.bfloat16))
+    assert ctx().poll() == 0
+    rk, rv = orc.compact_kv(k, v, idx)
+    got_k, got_v = bits_host(ko), bits_host(vo)
+    for h in range(hkv):
+        np.testing.assert_array_equal(got_k[:, h], rk[h])
+        np.testing.assert_array_equal(got_v[:, h], rv[h])
+    assert guards_intact(kfull, 0x1111) and guards_intact(vfull, 0x1111)
+
+
+def test_compact_rejects_in_place_and_bad_index():
+    n, hkv = 64, 2
+    k = bf16_dev(np.zeros((n, hkv, 128), np.uint16))
+    d = cc.Desc(hkv, hkv, 4, n=n, budget=8)
+    idx = torch.zeros((hkv, 8), dtype=torch.int32, device="cuda")
+    with pytest.raises(cc.CodecompError) as e:
+        cc.cc_compact_kv(ctx(), d, k, k, idx, k, k)
+    assert e.value.status == cc.CC_ERR_INVALID_ARG
+    idx[1, 3] = n + 7                                   # out of range: flagged and skipped
+    out = torch.zeros((8, hkv, 128), dtype=torch.bfloat16, device="cuda")
+    cc.cc_compact_kv(ctx(), d, k, k, idx, out, out.clone())
+    assert ctx().poll() == cc.CC_ERR_DEVICE_FLAG
+    assert ctx().poll() == 0                            # the status word is cleared by the poll
+
+
+def test_compact_paged():
+    wl = gen.Workload("p", 11, 1, 4, 2, 128, 8, gen.POOL_MAX, 3, 0, seq_lens=(100, 37, 260),
+                      budget_frac=0.25, page_size=16)
+    x = gen.make_layer(wl)
+    rng = np.random.Generator(np.random.PCG64(5))
+    buds = wl.budgets
+    b_tot = sum(buds)
+    idx = np.full((wl.n_heads_kv, b_tot), -1, np.int32)
+    off = 0
+    for s, (n, b) in enumerate(zip(wl.lens, buds)):
+        for h in range(wl.n_heads_kv):
+            idx[h, off:off + b] = np.sort(rng.choice(n, size=b, replace=False))
+        off += b
+    pt = torch.from_numpy(x.page_table).cuda()
+    stride = max((b + 15) // 16 for b in buds) + 2
+    d = desc_for(wl, cc.CC_MODE_FP32, page_table=pt, out_pt_stride=stride)
+    k_pool, v_pool = bf16_dev(x.k), bf16_dev(x.v)
+    before_k = bits_host(k_pool).copy()
+    out_pt = torch.full((len(buds), stride), -7, dtype=torch.int32, device="cuda")
+    cc.cc_compact_kv(ctx(), d, k_pool, v_pool, torch.from_numpy(idx).cuda(), k_pool, v_pool,
+                     torch.from_numpy(x.free_pages).cuda(), out_pt)
+    assert ctx().poll() == 0
+    pages = orc.assign_output_pages(buds, wl.lens, 16, x.free_pages)
+    got_pt = out_pt.cpu().numpy()
+    after_k, after_v = bits_host(k_pool), bits_host(v_pool)
+    off = 0
+    touched = np.zeros(x.pool_pages, bool)
+    for s, (n, b) in enumerate(zip(wl.lens, buds)):
+        assert got_pt[s, :len(pages[s])].tolist() == pages[s].tolist()
+        assert (got_pt[s, len(pages[s]):] == -1).all()
+        src = orc.paged_rows(x.page_table[s], n, 16)
+        dst = orc.paged_rows(pages[s], b, 16)
+        touched[pages[s]] = True
+        for h in range(wl.n_heads_kv):
+            tok = idx[h, off:off + b]
+            np.testing.assert_array_equal(after_k[dst, h], x.k[src[tok], h])
+            np.testing.assert_array_equal(after_v[dst, h], x.v[src[tok], h])
+        off += b
+    untouched_rows = np.repeat(~touched, 16)
+    np.testing.assert_array_equal(after_k[untouched_rows], before_k[untouched_rows])
+
+
+# ------------------------------------------------------------------ argument checks
+def test_descriptor_validation():
+    c = ctx()
+    ok = cc.Desc(8, 2, 32, n=128, budget=16)
+    assert c.workspace_bytes(ok) >= 256
+    for bad, status in [
+        (cc.Desc(8, 3, 32, n=128, budget=16), cc.CC_ERR_INVALID_ARG),
+        (cc.Desc(8, 2, 32, n=128, budget=16, head_dim=64), cc.CC_ERR_UNSUPPORTED),
+        (cc.Desc(8, 2, 32, n=128, budget=16, pool_size=4), cc.CC_ERR_UNSUPPORTED),
+        (cc.Desc(64, 1, 32, n=128, budget=16), cc.CC_ERR_UNSUPPORTED),          # w * G = 2048 rows
+        (cc.Desc(8, 2, 32, n=-1, budget=16), cc.CC_ERR_INVALID_ARG),
+        (cc.Desc(8, 2, 32, n=128, budget=16, page_size=12), cc.CC_ERR_UNSUPPORTED),
+    ]:
+        scores = torch.zeros(2, 128, device="cuda")
+        with pytest.raises(cc.CodecompError) as e:
+            cc.cc_fuse_prior_pool(c, bad, scores, scores[0], scores.clone())
+        assert e.value.status == status
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    big = cc.Desc(8, 2, 32, n=4096, budget=16)
+    with pytest.raises(cc.CodecompError) as e:
+        cc.cc_topk_select(c, big, torch.zeros(2, 4096, device="cuda"), torch.zeros(4096, device="cuda"),
+                          torch.zeros(2, 16, dtype=torch.int32, device="cuda"),
+                          torch.zeros(2, dtype=torch.int32, device="cuda"), ws=small)
+    assert e.value.status == cc.CC_ERR_WORKSPACE
