@@ -343,7 +343,8 @@ int cc_topk_select(cc_ctx* ctx, const cc_layer_desc* desc, const float* fused, c
   Plan p;
   int rc = build_plan(ctx, desc, &p);
   if (rc != CC_OK) return rc;
-  if (!fused || !prior || !idx || !count) return fail(ctx, CC_ERR_INVALID_ARG, "NULL tensor pointer");
+  if (!fused || !prior || !count || (!idx && p.bt.b_tot > 0))
+    return fail(ctx, CC_ERR_INVALID_ARG, "NULL tensor pointer");
   if ((rc = check_ws(ctx, p, ws, ws_bytes)) != CC_OK) return rc;
   return run_select(ctx, desc, p, fused, prior, idx, count, (char*)ws, stream);
 }
@@ -354,6 +355,7 @@ int cc_compact_kv(cc_ctx* ctx, const cc_layer_desc* desc, const void* k, const v
   Plan p;
   int rc = build_plan(ctx, desc, &p);
   if (rc != CC_OK) return rc;
+  if (p.bt.b_tot == 0) return CC_OK;
   if (!k || !v || !idx || !k_out || !v_out) return fail(ctx, CC_ERR_INVALID_ARG, "NULL tensor pointer");
   if ((uintptr_t)k % 16 || (uintptr_t)v % 16 || (uintptr_t)k_out % 16 || (uintptr_t)v_out % 16)
     return fail(ctx, CC_ERR_INVALID_ARG, "K/V pointers must be 16-byte aligned");
@@ -367,7 +369,7 @@ int cc_compress_layer(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win,
   Plan p;
   int rc = build_plan(ctx, desc, &p);
   if (rc != CC_OK) return rc;
-  if (!q_win || !k || !v || !prior || !k_out || !v_out || !idx || !count)
+  if (!q_win || !k || !v || !prior || !count || (p.bt.b_tot > 0 && (!k_out || !v_out || !idx)))
     return fail(ctx, CC_ERR_INVALID_ARG, "NULL tensor pointer");
   if ((uintptr_t)q_win % 16 || (uintptr_t)k % 16 || (uintptr_t)v % 16 || (uintptr_t)k_out % 16 ||
       (uintptr_t)v_out % 16)
@@ -379,6 +381,7 @@ int cc_compress_layer(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win,
   if ((rc = run_score(ctx, desc, p, q_win, k, scores, nullptr, w, stream)) != CC_OK) return rc;
   if ((rc = run_fuse(ctx, desc, p, scores, prior, fused, stream)) != CC_OK) return rc;
   if ((rc = run_select(ctx, desc, p, fused, prior, idx, count, w, stream)) != CC_OK) return rc;
+  if (p.bt.b_tot == 0) return CC_OK;
   return run_compact(ctx, desc, p, k, v, idx, k_out, v_out, free_pages, out_page_table, stream);
 }
 

@@ -146,10 +146,10 @@ score_simt_kernel(const __grid_constant__ BatchTable bt, const Geometry g, const
     }
     if (PASS == 2) {
       __syncthreads();
-      if (threadIdx.x < valid) {
+      for (int j = threadIdx.x; j < valid; j += blockDim.x) {
         float sum = 0.0f;
-        for (int wi = 0; wi < n_warps; ++wi) sum += colpart[wi][threadIdx.x];
-        a.scores[(int64_t)h * bt.n_tot + sq.tok_off + base + threadIdx.x] = sum;
+        for (int wi = 0; wi < n_warps; ++wi) sum += colpart[wi][j];
+        a.scores[(int64_t)h * bt.n_tot + sq.tok_off + base + j] = sum;
       }
     }
   }
