@@ -103,6 +103,7 @@ typedef struct cc_layer_desc {
   const int32_t* budgets;   /* HOST [num_seqs] */
   const int32_t* page_table;/* DEVICE [num_seqs][page_table_stride], used when page_size > 0 */
   int32_t page_table_stride;
+  int32_t pool_pages;       /* pages in the K/V pool (page ids must be < pool_pages) when page_size > 0 */
   int32_t out_page_table_stride; /* row length of out_page_table (>= ceil(B_s / page_size)) */
 } cc_layer_desc;
 

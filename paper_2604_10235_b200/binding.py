@@ -51,7 +51,8 @@ class cc_layer_desc(C.Structure):
         ("num_seqs", C.c_int32), ("page_size", C.c_int32),
         ("seq_lens", C.POINTER(C.c_int32)), ("budgets", C.POINTER(C.c_int32)),
         ("page_table", C.c_void_p),
-        ("page_table_stride", C.c_int32), ("out_page_table_stride", C.c_int32),
+        ("page_table_stride", C.c_int32), ("pool_pages", C.c_int32),
+        ("out_page_table_stride", C.c_int32),
     ]
 
 
@@ -154,7 +155,7 @@ class Desc:
                  compute_mode: int = CC_MODE_BF16, pool_kind: int = CC_POOL_MAX,
                  pool_size: int = 7, chunk_size: int = 1, alpha: float = 1.0, beta: float = 0.0,
                  force_threshold: float = math.inf, span_ratio: float = 0.0, span_min: int = 0,
-                 page_size: int = 0, page_table: Optional[torch.Tensor] = None,
+                 page_size: int = 0, page_table: Optional[torch.Tensor] = None, pool_pages: int = 0,
                  out_page_table_stride: int = 0, q_strides=None, kv_strides=None,
                  out_strides=(0, 0)):
         c = cc_layer_desc()
@@ -186,6 +187,7 @@ class Desc:
             self._keep.append(page_table)
             c.page_table = page_table.data_ptr()
             c.page_table_stride = page_table.shape[-1]
+        c.pool_pages = pool_pages
         c.out_page_table_stride = out_page_table_stride
         self.c = c
 

@@ -85,8 +85,8 @@ int build_plan(cc_ctx* ctx, const cc_layer_desc* d, Plan* p) {
     return fail(ctx, CC_ERR_UNSUPPORTED, "page_size must be 0, 8, 16, 32, 64 or 128");
   if (d->num_seqs > 0 && (!d->seq_lens || !d->budgets))
     return fail(ctx, CC_ERR_INVALID_ARG, "seq_lens / budgets are NULL");
-  if (ps > 0 && (!d->page_table || d->page_table_stride <= 0))
-    return fail(ctx, CC_ERR_INVALID_ARG, "paged layout needs page_table and its stride");
+  if (ps > 0 && (!d->page_table || d->page_table_stride <= 0 || d->pool_pages <= 0))
+    return fail(ctx, CC_ERR_INVALID_ARG, "paged layout needs page_table, its stride and pool_pages");
   if (d->q_stride_head % 8 || d->q_stride_row % 8 || d->q_stride_seq % 8 || d->kv_stride_tok % 8 ||
       d->kv_stride_head % 8 || d->out_stride_tok % 8 || d->out_stride_head % 8)
     return fail(ctx, CC_ERR_UNSUPPORTED, "strides must be multiples of 8 elements (16 bytes)");
@@ -190,7 +190,7 @@ int run_score(cc_ctx* ctx, const cc_layer_desc* d, const Plan& p, const void* q,
   }
   int drv = 0;
   cudaError_t e = launch_score_tc(L, p.bt, p.g, q, k, scores, lse, ws + p.off_score_ws,
-                                  ctx->encode_tiled, 0, &drv);
+                                  ctx->encode_tiled, (int64_t)d->pool_pages * d->page_size, &drv);
   if (drv != 0) return fail(ctx, CC_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", drv);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "score (tensor-core) launch");
   return CC_OK;

@@ -1,9 +1,699 @@
-// placeholder until the tensor-core kernel lands
+// A1, tensor-core mode (CC_MODE_BF16): window attention scores on sm_100a.
+//
+// u_h(j) = sum_r exp(s_rj - L_r) with s = q_r . k_j / sqrt(d) and L_r = log sum_j exp(s_rj),
+// where r runs over the w * G query rows that share KV head h.  L_r needs every key before
+// any column can be reduced, so the keys are streamed twice with the same persistent kernel:
+//
+//   pass 1  S = Q K^T with query rows on the MMA M axis: one TMEM lane, hence one thread, per
+//           query row, so the running maximum and sum of exp need no cross-thread traffic.
+//           Each CTA covers a contiguous span of key tiles and writes one (max, sum) pair per
+//           row; the spans of a (sequence, head) are merged in pass 2.
+//   pass 2  S^T = K Q^T with keys on the M axis: one thread per key, the query rows along the
+//           TMEM columns, so u(j) is a plain in-thread sum and is stored coalesced.
+//
+// Pipeline per CTA (one CTA per SM, 320 threads): warp 0 issues TMA loads (K tiles of 128 keys
+// through a ring of shared-memory stages, Q once per (sequence, head)), warp 1 issues
+// tcgen05.mma into two TMEM accumulator buffers, warps 2-9 drain the accumulators with
+// tcgen05.ld and do the exp / reduction work while the next tile is being multiplied.
+// All operands sit in shared memory in the 128-byte-swizzled K-major layout that both TMA
+// and the MMA descriptors understand; Q and K simply swap the A / B roles between passes.
+//
+// Every wait on an mbarrier is bounded: when the bound is hit the kernel records
+// CC_ERR_TIMEOUT, every role leaves its loop, TMEM is released and the kernel returns.
+#include <string.h>
+
 #include "cc_internal.cuh"
+
 namespace cc {
-size_t score_tc_ws_bytes(const BatchTable&, const Geometry&, int) { return 256; }
-cudaError_t launch_score_tc(const Launch&, const BatchTable&, const Geometry&, const void*,
-                            const void*, float*, float*, void*, void*, int64_t, int*) {
-  return cudaErrorNotSupported;
+
+namespace {
+
+constexpr int kThreads = 320;
+constexpr int kEpiWarps = 8;
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kMaxStages = 6;
+constexpr uint32_t kPanelBytes = kTileKeys * 128;        // one 64-channel half of a K tile
+constexpr uint32_t kStageBytes = 2 * kPanelBytes;        // 32 KB
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kBufCols = 256;                        // accumulator buffer stride
+constexpr uint32_t kMiscBytes = 8192;
+constexpr uint32_t kSmemLimit = 232448;                   // 227 KB
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+struct TcParams {
+  int grid;            // CTAs (same for both passes)
+  int total_tiles;     // H_kv * sum of tiles over the sequences
+  int rows;            // w * G
+  int rows_pad;        // G * w_pad, a multiple of 16
+  int w_pad;
+  int n_stages;
+  int n_sub;           // pass 1: 128-row blocks; pass 2: column chunks
+  int sub_cols;        // pass 2: rows per column chunk (multiple of 16, <= 256)
+  float2* part;        // [(grid + problems)][rows_pad] (max, sum) in the log2 domain
+  float* scores;
+  float* lse;
+  int64_t pool_rows;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok;
+}
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+               ::"r"(smem_dst), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols)
+               : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+               ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+        "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+        "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]),
+        "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
+        "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[8]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+        "=r"(v[7])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void epi_barrier() {      // the eight epilogue warps only
+  asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
+// 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);          // start address
+  d |= (uint64_t)1 << 16;                           // leading byte offset (unused with swizzle)
+  d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset
+  d |= (uint64_t)1 << 46;                           // descriptor version of sm_100
+  d |= (uint64_t)2 << 61;                           // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> f32, both operands K-major.
+__host__ __device__ constexpr uint32_t instr_desc(uint32_t m, uint32_t n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((m >> 4) << 24);
+}
+
+// ------------------------------------------------------------------ shared state
+struct Barriers {
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
+  uint64_t q_full, q_empty;
+  uint64_t acc_full[2], acc_empty[2];
+};
+
+struct Misc {                        // lives in the last kMiscBytes of dynamic shared memory
+  float neg_lc[kMaxRows];            // pass 2: -L_r in the log2 domain (+inf rows give 0)
+  float2 xchg[kMaxRows];             // pass 1: (max, sum) hand-over; pass 2: partial u (as .x)
+  Barriers bar;
+  uint32_t tmem_base;
+  volatile int abort_flag;
+};
+static_assert(sizeof(Misc) <= kMiscBytes, "Misc does not fit");
+
+struct Pipe {
+  Misc* misc;
+  DeviceStatus* status;
+};
+
+// Bounded wait; false (and the abort flag set) when the bound is hit or another role gave up.
+__device__ __forceinline__ bool wait_bar(const Pipe& p, uint64_t* bar, uint32_t parity, int where) {
+  const uint32_t b = smem_u32(bar);
+  for (uint32_t i = 0; i < 4000000u; ++i) {
+    if (mbar_try_wait(b, parity)) return true;
+    if (p.misc->abort_flag) return false;
+    if (i > 2048) __nanosleep(64);
+  }
+  p.misc->abort_flag = 1;
+  report_error(p.status, CC_ERR_TIMEOUT, where);
+  return false;
+}
+
+// Walks the tiles of a CTA's span in (sequence, head, tile) order.
+struct TileCursor {
+  int s, h, local, n_tiles;
+  __device__ void locate(const BatchTable& bt, int hkv, int t) {
+    for (s = 0; s < bt.num_seqs; ++s) {
+      const int lo = hkv * bt.seq[s].tile_off, cnt = hkv * bt.seq[s].n_tiles;
+      if (t < lo + cnt) {
+        n_tiles = bt.seq[s].n_tiles;
+        h = (t - lo) / n_tiles;
+        local = (t - lo) % n_tiles;
+        return;
+      }
+    }
+    s = bt.num_seqs - 1; h = 0; local = 0; n_tiles = 1;   // not reached for t < total_tiles
+  }
+  __device__ void advance(const BatchTable& bt, int hkv) {
+    if (++local < n_tiles) return;
+    local = 0;
+    if (++h < hkv) return;
+    h = 0;
+    do { ++s; } while (s < bt.num_seqs && bt.seq[s].n_tiles == 0);
+    n_tiles = s < bt.num_seqs ? bt.seq[s].n_tiles : 1;
+  }
+  __device__ int problem(int hkv) const { return s * hkv + h; }
+};
+
+__device__ __forceinline__ int span_begin(int b, const TcParams& P) {
+  return (int)(((long long)b * P.total_tiles) / P.grid);
+}
+__device__ __forceinline__ int cta_of_tile(int t, const TcParams& P) {
+  return (int)((((long long)t + 1) * P.grid - 1) / P.total_tiles);
+}
+
+// ------------------------------------------------------------------ the kernel
+template <int PASS>
+__global__ void __launch_bounds__(kThreads, 1)
+score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ Geometry g,
+                const __grid_constant__ TcParams P, const __grid_constant__ CUtensorMap q_map,
+                const __grid_constant__ CUtensorMap k_map, DeviceStatus* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t q_bytes = (uint32_t)P.rows_pad * 256u;
+  const uint32_t q_panel = (uint32_t)P.rows_pad * 128u;
+  uint8_t* q_smem = smem;
+  uint8_t* k_smem = smem + q_bytes;
+  Misc* misc = reinterpret_cast<Misc*>(k_smem + (size_t)P.n_stages * kStageBytes);
+  Pipe pipe{misc, status};
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t_begin = span_begin(blockIdx.x, P), t_end = span_begin(blockIdx.x + 1, P);
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kMaxStages; ++i) {
+      mbar_init(smem_u32(&misc->bar.full[i]), 1);
+      mbar_init(smem_u32(&misc->bar.empty[i]), 1);
+    }
+    mbar_init(smem_u32(&misc->bar.q_full), 1);
+    mbar_init(smem_u32(&misc->bar.q_empty), 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&misc->bar.acc_full[i]), 1);
+      mbar_init(smem_u32(&misc->bar.acc_empty[i]), kEpiWarps);
+    }
+    misc->abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&misc->tmem_base), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = misc->tmem_base;
+
+  if (warp == 0) {
+    // ================================================================ TMA producer
+    if (lane == 0) {
+      TileCursor cur;
+      cur.locate(bt, g.hkv, t_begin);
+      int stage = 0, cur_problem = -1;
+      uint32_t phase = 0, qe_phase = 0;
+      for (int t = t_begin; t < t_end; ++t, cur.advance(bt, g.hkv)) {
+        const SeqInfo& sq = bt.seq[cur.s];
+        if (cur.problem(g.hkv) != cur_problem) {
+          if (cur_problem >= 0) {
+            if (!wait_bar(pipe, &misc->bar.q_empty, qe_phase, 10)) break;
+            qe_phase ^= 1;
+          }
+          cur_problem = cur.problem(g.hkv);
+          const uint32_t qb = smem_u32(&misc->bar.q_full);
+          mbar_expect_tx(qb, q_bytes);
+          tma_load_4d(smem_u32(q_smem), &q_map, qb, 0, cur.h * g.group, 0, cur.s);
+          tma_load_4d(smem_u32(q_smem) + q_panel, &q_map, qb, 64, cur.h * g.group, 0, cur.s);
+        }
+        if (!wait_bar(pipe, &misc->bar.empty[stage], phase ^ 1, 11)) break;
+        const uint32_t fb = smem_u32(&misc->bar.full[stage]);
+        const uint32_t dst = smem_u32(k_smem) + (uint32_t)stage * kStageBytes;
+        const int key0 = cur.local * kTileKeys;
+        if (bt.page_size == 0) {
+          mbar_expect_tx(fb, kStageBytes);
+          tma_load_3d(dst, &k_map, fb, 0, cur.h, sq.tok_off + key0);
+          tma_load_3d(dst + kPanelBytes, &k_map, fb, 64, cur.h, sq.tok_off + key0);
+        } else {
+          const int ps = bt.page_size;
+          const int valid = min(kTileKeys, sq.n - key0);
+          const int n_pages = (valid + ps - 1) / ps;
+          const int32_t* pt = g.page_table + (int64_t)cur.s * g.page_table_stride + key0 / ps;
+          int ids[16];
+          int good = 0;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            ids[i] = -1;
+            if (i < n_pages) {
+              ids[i] = pt[i];
+              if (ids[i] < 0 || ((int64_t)ids[i] + 1) * ps > P.pool_rows) {
+                ids[i] = -1;
+                report_error(status, CC_ERR_DEVICE_FLAG, 12);
+              } else {
+                ++good;
+              }
+            }
+          }
+          mbar_expect_tx(fb, (uint32_t)good * (uint32_t)ps * 256u);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            if (ids[i] >= 0) {
+              const uint32_t off = (uint32_t)i * (uint32_t)ps * 128u;
+              tma_load_3d(dst + off, &k_map, fb, 0, cur.h, ids[i] * ps);
+              tma_load_3d(dst + kPanelBytes + off, &k_map, fb, 64, cur.h, ids[i] * ps);
+            }
+          }
+        }
+        if (++stage == P.n_stages) { stage = 0; phase ^= 1; }
+      }
+    }
+  } else if (warp == 1) {
+    // ================================================================ MMA issuer
+    if (lane == 0) {
+      TileCursor cur;
+      cur.locate(bt, g.hkv, t_begin);
+      int stage = 0, cur_problem = -1;
+      uint32_t phase = 0, qf_phase = 0, item = 0;
+      const uint32_t q_addr = smem_u32(q_smem);
+      bool ok = true;
+      for (int t = t_begin; t < t_end && ok; ++t) {
+        if (cur.problem(g.hkv) != cur_problem) {
+          cur_problem = cur.problem(g.hkv);
+          if (!wait_bar(pipe, &misc->bar.q_full, qf_phase, 20)) break;
+          qf_phase ^= 1;
+        }
+        if (!wait_bar(pipe, &misc->bar.full[stage], phase, 21)) break;
+        tc_fence_after();
+        const uint32_t k_addr = smem_u32(k_smem) + (uint32_t)stage * kStageBytes;
+        for (int sub = 0; sub < P.n_sub; ++sub, ++item) {
+          const uint32_t buf = item & 1u;
+          if (!wait_bar(pipe, &misc->bar.acc_empty[buf], ((item >> 1) & 1u) ^ 1u, 22)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + buf * kBufCols;
+          uint32_t idesc, q_off;
+          if (PASS == 1) {
+            idesc = instr_desc(128, kTileKeys);
+            q_off = (uint32_t)sub * 128u * 128u;                 // 128-row block of Q
+          } else {
+            const int c0 = sub * P.sub_cols;
+            const int nc = min(P.sub_cols, P.rows_pad - c0);
+            idesc = instr_desc(128, (uint32_t)nc);
+            q_off = (uint32_t)c0 * 128u;
+          }
+#pragma unroll
+          for (int ks = 0; ks < kHeadDim / 16; ++ks) {
+            const uint32_t inner = (uint32_t)(ks & 3) * 32u;
+            const uint64_t qd = smem_desc(q_addr + (ks >> 2) * q_panel + q_off + inner);
+            const uint64_t kd = smem_desc(k_addr + (ks >> 2) * kPanelBytes + inner);
+            if (PASS == 1) umma_bf16(d_tmem, qd, kd, idesc, ks > 0);
+            else           umma_bf16(d_tmem, kd, qd, idesc, ks > 0);
+          }
+          umma_commit(smem_u32(&misc->bar.acc_full[buf]));
+        }
+        if (!ok) break;
+        umma_commit(smem_u32(&misc->bar.empty[stage]));
+        if (++stage == P.n_stages) { stage = 0; phase ^= 1; }
+        const int prev_problem = cur.problem(g.hkv);
+        cur.advance(bt, g.hkv);
+        if (t + 1 < t_end && cur.problem(g.hkv) != prev_problem)
+          umma_commit(smem_u32(&misc->bar.q_empty));
+      }
+    }
+  } else {
+    // ================================================================ epilogue warps
+    const int ew = warp - 2;                 // 0..7
+    const int quad = warp & 3;               // TMEM lane quadrant this warp may read
+    const int half = ew >> 2;                // which half of the columns
+    const int row_in_tile = quad * 32 + lane;
+    const int etid = half * 128 + row_in_tile;            // 0..255, unique per epilogue thread
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+    const float c = kLog2e / sqrtf((float)kHeadDim);
+    TileCursor cur;
+    cur.locate(bt, g.hkv, t_begin);
+    int cur_problem = -1, cur_s = 0, cur_h = 0;
+    uint32_t item = 0;
+    bool dead = false;      // after a failed wait: keep the loop structure (and its barriers), skip the work
+    float run_m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+    float run_l[4] = {0.f, 0.f, 0.f, 0.f};
+
+    // pass 1: hand the two column halves' (max, sum) together and write the span's partial
+    auto flush_partial = [&](int problem) {
+#pragma unroll
+      for (int rb = 0; rb < 4; ++rb) {
+        if (rb >= P.n_sub) break;
+        const int row = rb * 128 + row_in_tile;
+        if (half == 1) misc->xchg[row] = make_float2(run_m[rb], run_l[rb]);
+      }
+      epi_barrier();
+#pragma unroll
+      for (int rb = 0; rb < 4; ++rb) {
+        if (rb >= P.n_sub) break;
+        const int row = rb * 128 + row_in_tile;
+        if (half == 0 && row < P.rows_pad) {
+          const float2 o = misc->xchg[row];
+          const float m = fmaxf(run_m[rb], o.x);
+          float l = 0.f;
+          if (m > -INFINITY) l = run_l[rb] * ex2(run_m[rb] - m) + o.y * ex2(o.x - m);
+          P.part[(int64_t)(blockIdx.x + problem) * P.rows_pad + row] = make_float2(m, l);
+        }
+        run_m[rb] = -INFINITY;
+        run_l[rb] = 0.f;
+      }
+      epi_barrier();
+    };
+
+    for (int t = t_begin; t < t_end; ++t, cur.advance(bt, g.hkv)) {
+      const SeqInfo& sq = bt.seq[cur.s];
+      if (cur.problem(g.hkv) != cur_problem) {
+        if (PASS == 1) {
+          if (cur_problem >= 0) flush_partial(cur_problem);
+        } else {
+          // merge the spans' (max, sum) of the new (sequence, head) into -L_r
+          epi_barrier();
+          const int first_tile = g.hkv * sq.tile_off + cur.h * sq.n_tiles;
+          const int b0 = cta_of_tile(first_tile, P), b1 = cta_of_tile(first_tile + sq.n_tiles - 1, P);
+          const int problem = cur.problem(g.hkv);
+          for (int row = etid; row < P.rows_pad; row += kEpiThreads) {
+            float m = -INFINITY;
+            for (int b = b0; b <= b1; ++b)
+              m = fmaxf(m, P.part[(int64_t)(b + problem) * P.rows_pad + row].x);
+            float l = 0.f;
+            for (int b = b0; b <= b1; ++b) {
+              const float2 pr = P.part[(int64_t)(b + problem) * P.rows_pad + row];
+              if (pr.y > 0.f) l += pr.y * ex2(pr.x - m);
+            }
+            const float lc = m + log2f(l);
+            const int gq = row % g.group, tq = row / g.group;     // row = t * G + g
+            const bool real = tq < g.window;
+            misc->neg_lc[row] = real ? -lc : -INFINITY;
+            if (real && P.lse != nullptr && t == first_tile)
+              P.lse[((int64_t)cur.s * g.hq + cur.h * g.group + gq) * g.window + tq] = lc * kLn2;
+          }
+          epi_barrier();
+        }
+        cur_problem = cur.problem(g.hkv);
+        cur_s = cur.s;
+        cur_h = cur.h;
+      }
+      const int key0 = cur.local * kTileKeys;
+      const int valid = min(kTileKeys, sq.n - key0);
+      float u_acc = 0.f;
+
+#pragma unroll 1
+      for (int sub = 0; sub < P.n_sub; ++sub, ++item) {
+        const uint32_t buf = item & 1u;
+        if (!dead) {
+          const bool got = wait_bar(pipe, &misc->bar.acc_full[buf], (item >> 1) & 1u, 30);
+          dead = !__all_sync(0xffffffffu, got);
+        }
+        if (dead) continue;
+        tc_fence_after();
+        const uint32_t acc_addr = lane_addr + buf * kBufCols;
+        if (PASS == 1) {
+          // thread = query row (sub * 128 + row_in_tile); columns = keys of this half
+          const int col_lo = half * (kTileKeys / 2);
+          float m_run = -INFINITY, l_run = 0.f;
+#pragma unroll
+          for (int rb = 0; rb < 4; ++rb) if (rb == sub) { m_run = run_m[rb]; l_run = run_l[rb]; }
+#pragma unroll 1
+          for (int cc0 = 0; cc0 < kTileKeys / 2; cc0 += 32) {
+            uint32_t v[32];
+            tmem_ld32(acc_addr + (uint32_t)(col_lo + cc0), v);
+            tmem_wait_ld();
+            float mx = -INFINITY;
+            if (valid == kTileKeys) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                if (col_lo + cc0 + i >= valid) v[i] = 0xff800000u;       // -inf
+                mx = fmaxf(mx, __uint_as_float(v[i]));
+              }
+            }
+            const float m_new = fmaxf(m_run, mx * c);
+            if (m_new > -INFINITY) {
+              float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+              for (int i = 0; i < 32; i += 4) {
+                a0 += ex2(fmaf(__uint_as_float(v[i + 0]), c, -m_new));
+                a1 += ex2(fmaf(__uint_as_float(v[i + 1]), c, -m_new));
+                a2 += ex2(fmaf(__uint_as_float(v[i + 2]), c, -m_new));
+                a3 += ex2(fmaf(__uint_as_float(v[i + 3]), c, -m_new));
+              }
+              l_run = l_run * ex2(m_run - m_new) + ((a0 + a1) + (a2 + a3));
+              m_run = m_new;
+            }
+          }
+#pragma unroll
+          for (int rb = 0; rb < 4; ++rb) if (rb == sub) { run_m[rb] = m_run; run_l[rb] = l_run; }
+        } else {
+          // thread = key (key0 + row_in_tile); columns = query rows of this chunk's half
+          const int c0 = sub * P.sub_cols;
+          const int nc = min(P.sub_cols, P.rows_pad - c0);
+          const int hc = nc >> 1;                         // multiple of 8
+          const int col_lo = half * hc;
+          const float* nl = misc->neg_lc + c0 + col_lo;
+          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+          int cc0 = 0;
+#pragma unroll 1
+          for (; cc0 + 32 <= hc; cc0 += 32) {
+            uint32_t v[32];
+            tmem_ld32(acc_addr + (uint32_t)(col_lo + cc0), v);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+              const float4 L = *reinterpret_cast<const float4*>(nl + cc0 + i);
+              a0 += ex2(fmaf(__uint_as_float(v[i + 0]), c, L.x));
+              a1 += ex2(fmaf(__uint_as_float(v[i + 1]), c, L.y));
+              a2 += ex2(fmaf(__uint_as_float(v[i + 2]), c, L.z));
+              a3 += ex2(fmaf(__uint_as_float(v[i + 3]), c, L.w));
+            }
+          }
+#pragma unroll 1
+          for (; cc0 < hc; cc0 += 8) {
+            uint32_t v[8];
+            tmem_ld8(acc_addr + (uint32_t)(col_lo + cc0), v);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 8; i += 4) {
+              const float4 L = *reinterpret_cast<const float4*>(nl + cc0 + i);
+              a0 += ex2(fmaf(__uint_as_float(v[i + 0]), c, L.x));
+              a1 += ex2(fmaf(__uint_as_float(v[i + 1]), c, L.y));
+              a2 += ex2(fmaf(__uint_as_float(v[i + 2]), c, L.z));
+              a3 += ex2(fmaf(__uint_as_float(v[i + 3]), c, L.w));
+            }
+          }
+          u_acc += (a0 + a1) + (a2 + a3);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&misc->bar.acc_empty[buf]));
+      }
+      if (PASS == 2) {
+        // the two column halves of a key meet through shared memory (double buffered by tile)
+        float* xu = reinterpret_cast<float*>(misc->xchg) + (t & 1) * kTileKeys;
+        if (half == 1) xu[row_in_tile] = u_acc;
+        epi_barrier();
+        if (!dead && half == 0 && row_in_tile < valid)
+          P.scores[(int64_t)cur_h * bt.n_tot + bt.seq[cur_s].tok_off + key0 + row_in_tile] =
+              u_acc + xu[row_in_tile];
+      }
+    }
+    if (PASS == 1 && cur_problem >= 0) flush_partial(cur_problem);
+  }
+
+  // ---------------------------------------------------------------- teardown
+  if (misc->abort_flag) {
+    // give copies still in flight time to land before shared memory is released
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TcPlan {
+  TcParams P;
+  size_t smem_bytes;
+  bool ok;
+};
+
+TcPlan make_plan(const BatchTable& bt, const Geometry& g, int sm_count) {
+  TcPlan pl;
+  TcParams& P = pl.P;
+  memset(&pl, 0, sizeof(pl));
+  P.total_tiles = g.hkv * bt.tiles_per_head;
+  P.grid = P.total_tiles < sm_count ? P.total_tiles : sm_count;
+  if (P.grid < 1) P.grid = 1;
+  P.rows = g.rows;
+  // pad the window so that the padded row count is a multiple of 16 (UMMA N granularity)
+  int w_pad = g.window;
+  while ((g.group * w_pad) % 16 != 0) ++w_pad;
+  P.w_pad = w_pad;
+  P.rows_pad = g.group * w_pad;
+  pl.ok = P.rows_pad <= kMaxRows && w_pad <= 256 && g.group <= 256;
+  const uint32_t q_bytes = (uint32_t)P.rows_pad * 256u;
+  int stages = ((int)kSmemLimit - 1024 - (int)kMiscBytes - (int)q_bytes) / (int)kStageBytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < 2) pl.ok = false;
+  P.n_stages = stages;
+  pl.smem_bytes = 1024 + q_bytes + (size_t)stages * kStageBytes + kMiscBytes;
+  return pl;
+}
+
+}  // namespace
+
+size_t score_tc_ws_bytes(const BatchTable& bt, const Geometry& g, int sm_count) {
+  TcPlan pl = make_plan(bt, g, sm_count);
+  const size_t entries = (size_t)pl.P.grid + (size_t)bt.num_seqs * g.hkv;
+  return (entries * pl.P.rows_pad * sizeof(float2) + 255) / 256 * 256;
+}
+
+cudaError_t launch_score_tc(const Launch& L, const BatchTable& bt, const Geometry& g,
+                            const void* q, const void* k, float* scores, float* lse, void* ws,
+                            void* encode_fn, int64_t pool_rows, int* drv_err) {
+  *drv_err = 0;
+  TcPlan pl = make_plan(bt, g, L.sm_count);
+  if (!pl.ok) return cudaErrorInvalidConfiguration;
+  TcParams& P = pl.P;
+  P.part = (float2*)ws;
+  P.scores = scores;
+  P.lse = lse;
+  P.pool_rows = bt.page_size > 0 ? pool_rows : (int64_t)bt.n_tot;
+
+  EncodeTiledFn encode = (EncodeTiledFn)encode_fn;
+  CUtensorMap q_map, k_map;
+  {
+    const int S = bt.num_seqs;
+    cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)g.hq, (cuuint64_t)g.window, (cuuint64_t)S};
+    int64_t seq_stride = g.q_stride_seq;
+    if (S == 1 || seq_stride <= 0) seq_stride = g.q_stride_row * g.window;
+    cuuint64_t strides[3] = {(cuuint64_t)g.q_stride_head * 2, (cuuint64_t)g.q_stride_row * 2,
+                             (cuuint64_t)seq_stride * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)g.group, (cuuint32_t)P.w_pad, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = encode(&q_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(q), dims,
+                        strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { *drv_err = (int)r; return cudaErrorUnknown; }
+  }
+  {
+    cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)g.hkv, (cuuint64_t)P.pool_rows};
+    cuuint64_t strides[2] = {(cuuint64_t)g.kv_stride_head * 2, (cuuint64_t)g.kv_stride_tok * 2};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)(bt.page_size > 0 ? bt.page_size : kTileKeys)};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = encode(&k_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(k), dims,
+                        strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { *drv_err = (int)r; return cudaErrorUnknown; }
+  }
+
+  cudaError_t e;
+  e = cudaFuncSetAttribute(score_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)pl.smem_bytes);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(score_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)pl.smem_bytes);
+  if (e != cudaSuccess) return e;
+
+  P.n_sub = (P.rows_pad + 127) / 128;
+  P.sub_cols = 0;
+  score_tc_kernel<1><<<P.grid, kThreads, pl.smem_bytes, L.stream>>>(bt, g, P, q_map, k_map, L.status);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+
+  P.n_sub = (P.rows_pad + 255) / 256;
+  P.sub_cols = ((P.rows_pad + P.n_sub - 1) / P.n_sub + 15) / 16 * 16;
+  score_tc_kernel<2><<<P.grid, kThreads, pl.smem_bytes, L.stream>>>(bt, g, P, q_map, k_map, L.status);
+  return cudaGetLastError();
+}
+
 }  // namespace cc

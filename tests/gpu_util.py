@@ -33,12 +33,13 @@ def f32_dev(x) -> torch.Tensor:
 
 
 def desc_for(wl: gen.Workload, mode: int, page_table=None, out_pt_stride: int = 0,
-             force: bool = True) -> cc.Desc:
+             force: bool = True, pool_pages: int = 0) -> cc.Desc:
     kw = dict(head_dim=wl.head_dim, compute_mode=mode, pool_kind=wl.pool_kind,
               pool_size=wl.pool_size, chunk_size=wl.chunk_size, alpha=wl.alpha, beta=wl.beta,
               force_threshold=wl.force_threshold if force else math.inf,
               span_ratio=wl.span_ratio, span_min=wl.span_min, page_size=wl.page_size,
-              page_table=page_table, out_page_table_stride=out_pt_stride)
+              page_table=page_table, out_page_table_stride=out_pt_stride,
+              pool_pages=pool_pages)
     if wl.seq_lens:
         return cc.Desc(wl.n_heads_q, wl.n_heads_kv, wl.window, seq_lens=wl.lens,
                        budgets=wl.budgets, **kw)

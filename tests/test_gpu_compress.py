@@ -24,7 +24,7 @@ def run_layer(wl, x, mode):
     buds, lens = wl.budgets, wl.lens
     b_tot = sum(buds)
     stride = max((min(b, n) + wl.page_size - 1) // wl.page_size for b, n in zip(buds, lens)) + 1 if paged else 0
-    d = desc_for(wl, mode, page_table=pt, out_pt_stride=stride)
+    d = desc_for(wl, mode, page_table=pt, out_pt_stride=stride, pool_pages=x.pool_pages)
     k, v = bf16_dev(x.k), bf16_dev(x.v)
     idx = torch.full((wl.n_heads_kv, b_tot), -9, dtype=torch.int32, device="cuda")
     count = torch.full((len(lens), wl.n_heads_kv), -9, dtype=torch.int32, device="cuda")

@@ -17,7 +17,7 @@ MODES = [(cc.CC_MODE_FP32, 1e-5), (cc.CC_MODE_BF16, 2e-3)]
 
 def run_scores(wl, x, mode, want_lse=True):
     pt = torch.from_numpy(x.page_table).cuda() if wl.page_size else None
-    d = desc_for(wl, mode, page_table=pt)
+    d = desc_for(wl, mode, page_table=pt, pool_pages=x.pool_pages)
     n_tot = sum(wl.lens)
     scores = torch.full((wl.n_heads_kv, n_tot), -1.0, device="cuda")
     lse = torch.full((len(wl.lens), wl.n_heads_q, wl.window), -1.0, device="cuda") if want_lse else None

@@ -216,7 +216,7 @@ def test_compact_paged():
         off += b
     pt = torch.from_numpy(x.page_table).cuda()
     stride = max((b + 15) // 16 for b in buds) + 2
-    d = desc_for(wl, cc.CC_MODE_FP32, page_table=pt, out_pt_stride=stride)
+    d = desc_for(wl, cc.CC_MODE_FP32, page_table=pt, out_pt_stride=stride, pool_pages=x.pool_pages)
     k_pool, v_pool = bf16_dev(x.k), bf16_dev(x.v)
     before_k = bits_host(k_pool).copy()
     out_pt = torch.full((len(buds), stride), -7, dtype=torch.int32, device="cuda")
