@@ -1,0 +1,93 @@
+"""User-facing wrapper: compress one layer's KV cache starting from host or device tensors.
+
+``LayerCompressor`` owns the device buffers (inputs, outputs, workspace) for one layer
+geometry so that repeated calls allocate nothing, and forwards to ``cc_compress_layer``.
+All arithmetic happens in libcodecomp's kernels; this file only moves bytes.
+"""
+from __future__ import annotations
+
+from typing import Dict, Optional
+
+import numpy as np
+import torch
+
+from . import binding as cc
+from . import inputs as gen
+
+
+def desc_from_workload(wl: gen.Workload, mode: int = cc.CC_MODE_BF16,
+                       page_table: Optional[torch.Tensor] = None, pool_pages: int = 0,
+                       out_pt_stride: int = 0) -> cc.Desc:
+    kw = dict(head_dim=wl.head_dim, compute_mode=mode, pool_kind=wl.pool_kind,
+              pool_size=wl.pool_size, chunk_size=wl.chunk_size, alpha=wl.alpha, beta=wl.beta,
+              force_threshold=wl.force_threshold, span_ratio=wl.span_ratio, span_min=wl.span_min,
+              page_size=wl.page_size, page_table=page_table, pool_pages=pool_pages,
+              out_page_table_stride=out_pt_stride)
+    if wl.seq_lens:
+        return cc.Desc(wl.n_heads_q, wl.n_heads_kv, wl.window, seq_lens=wl.lens,
+                       budgets=wl.budgets, **kw)
+    return cc.Desc(wl.n_heads_q, wl.n_heads_kv, wl.window, n=wl.n, budget=wl.budget, **kw)
+
+
+def to_bf16(bits: np.ndarray, device: str = "cuda", pin: bool = False) -> torch.Tensor:
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16)
+    if device == "cpu":
+        return t.pin_memory() if pin else t
+    return t.to(device)
+
+
+class LayerCompressor:
+    """Pre-allocated state for repeated ``cc_compress_layer`` calls on one geometry
+    (contiguous K/V layout)."""
+
+    def __init__(self, ctx: cc.Context, wl: gen.Workload, mode: int = cc.CC_MODE_BF16):
+        assert wl.page_size == 0, "LayerCompressor handles the contiguous layout"
+        self.ctx, self.wl = ctx, wl
+        self.desc = desc_from_workload(wl, mode)
+        dev = f"cuda:{ctx.device}"
+        S, hq, hkv, d = len(wl.lens), wl.n_heads_q, wl.n_heads_kv, wl.head_dim
+        n_tot, b_tot = self.desc.n_tot, self.desc.b_tot
+        bf = torch.bfloat16
+        self.q = torch.empty((S, wl.window, hq, d), dtype=bf, device=dev)
+        self.k = torch.empty((n_tot, hkv, d), dtype=bf, device=dev)
+        self.v = torch.empty((n_tot, hkv, d), dtype=bf, device=dev)
+        self.prior = torch.empty((n_tot,), dtype=torch.float32, device=dev)
+        self.k_out = torch.empty((b_tot, hkv, d), dtype=bf, device=dev)
+        self.v_out = torch.empty((b_tot, hkv, d), dtype=bf, device=dev)
+        self.idx = torch.empty((hkv, b_tot), dtype=torch.int32, device=dev)
+        self.count = torch.empty((S, hkv), dtype=torch.int32, device=dev)
+        self.ws = ctx.workspace(self.desc)
+        # pinned landing buffers for the results
+        self.h_k_out = torch.empty(self.k_out.shape, dtype=bf).pin_memory()
+        self.h_v_out = torch.empty(self.v_out.shape, dtype=bf).pin_memory()
+        self.h_idx = torch.empty(self.idx.shape, dtype=torch.int32).pin_memory()
+        self.h_count = torch.empty(self.count.shape, dtype=torch.int32).pin_memory()
+
+    @property
+    def h2d_bytes(self) -> int:
+        return sum(t.numel() * t.element_size() for t in (self.q, self.k, self.v, self.prior))
+
+    @property
+    def d2h_bytes(self) -> int:
+        return sum(t.numel() * t.element_size()
+                   for t in (self.k_out, self.v_out, self.idx, self.count))
+
+    def run_device(self, q, k, v, prior) -> None:
+        """Inputs already on the device; outputs land in self.k_out / v_out / idx / count."""
+        cc.cc_compress_layer(self.ctx, self.desc, q, k, v, prior, self.k_out, self.v_out,
+                             self.idx, self.count, ws=self.ws)
+
+    def run_host(self, q_h, k_h, v_h, prior_h) -> Dict[str, torch.Tensor]:
+        """Inputs in (pinned) host memory: copy in, compress, copy the compacted cache back.
+        Everything is enqueued on the current stream; the caller synchronises."""
+        self.q.copy_(q_h, non_blocking=True)
+        self.k.copy_(k_h, non_blocking=True)
+        self.v.copy_(v_h, non_blocking=True)
+        self.prior.copy_(prior_h, non_blocking=True)
+        self.run_device(self.q, self.k, self.v, self.prior)
+        self.h_k_out.copy_(self.k_out, non_blocking=True)
+        self.h_v_out.copy_(self.v_out, non_blocking=True)
+        self.h_idx.copy_(self.idx, non_blocking=True)
+        self.h_count.copy_(self.count, non_blocking=True)
+        return {"k_out": self.h_k_out, "v_out": self.h_v_out, "idx": self.h_idx,
+                "count": self.h_count}
