@@ -151,6 +151,24 @@ int cc_topk_select(cc_ctx* ctx, const cc_layer_desc* desc, const float* fused,
                    const float* prior, int32_t* idx, int32_t* count,
                    void* ws, size_t ws_bytes, void* stream);
 
+/* (No counterpart in the paper.)  The same selection as cc_topk_select for callers that cannot
+ * hand the library a workspace because they cannot allocate device memory at that point: a
+ * serving process whose memory pool already owns the whole device, or a step of a request
+ * loop where cudaMalloc - which may block until the device is idle - is not acceptable.  The
+ * one scratch array the kernel needs (a flag byte per head and item) lives in a fixed array
+ * inside the library's device image: CC_STATIC_SELECT_MAX_ITEMS bytes on every GPU that loads
+ * the library, held until the process exits.  Calls with n_heads_kv * (total items of the
+ * batch) above that limit fail with CC_ERR_UNSUPPORTED and enqueue nothing.  The call
+ * allocates and frees nothing.  Its first use on a device looks up the array's device address
+ * (the context's device must be the current device); make that first call outside any stream
+ * capture.  All calls, from every context and stream, share the one array: two calls whose
+ * kernels may run at the same time on the GPU race, so keep them ordered (one stream, or
+ * events).  Nothing needs clearing between calls: every flag is written before it is read.
+ * Inputs and outputs are exactly those of cc_topk_select. */
+#define CC_STATIC_SELECT_MAX_ITEMS (1 << 20)
+int cc_topk_select_static(cc_ctx* ctx, const cc_layer_desc* desc, const float* fused,
+                          const float* prior, int32_t* idx, int32_t* count, void* stream);
+
 /* A5 - compaction: k_out[slot i of head h] = k[token idx[h][i] of head h], same for v, as
  * bit copies.  Paged layout: sequence s receives ceil(min(B_s, n_s) / page_size) page ids,
  * taken in order from free_pages (device i32, sequences served in order), written to

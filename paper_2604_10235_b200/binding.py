@@ -28,7 +28,8 @@ CC_MAX_SEQS = 64
 
 EXPORTS = ("cc_create", "cc_destroy", "cc_status_string", "cc_last_error", "cc_poll_status",
            "cc_workspace_bytes", "cc_score_window", "cc_fuse_prior_pool", "cc_topk_select",
-           "cc_compact_kv", "cc_compress_layer", "cc_workspace_views")
+           "cc_compact_kv", "cc_compress_layer", "cc_workspace_views", "cc_topk_select_static")
+CC_STATIC_SELECT_MAX_ITEMS = 1 << 20
 
 
 class CodecompError(RuntimeError):
@@ -87,6 +88,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.cc_score_window.argtypes = [vp, dp, vp, vp, vp, vp, vp, sz, vp]
     lib.cc_fuse_prior_pool.argtypes = [vp, dp, vp, vp, vp, vp]
     lib.cc_topk_select.argtypes = [vp, dp, vp, vp, vp, vp, vp, sz, vp]
+    lib.cc_topk_select_static.argtypes = [vp, dp, vp, vp, vp, vp, vp]
     lib.cc_compact_kv.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.cc_compress_layer.argtypes = [vp, dp] + [vp] * 10 + [vp, sz, vp]
     lib.cc_workspace_views.argtypes = [vp, dp, vp, C.POINTER(vp), C.POINTER(vp)]
@@ -245,6 +247,16 @@ def cc_topk_select(ctx: Context, desc: Desc, fused, prior, idx, count, ws=None, 
     ctx.check(ctx.lib.cc_topk_select(ctx.handle, C.byref(desc.c), _ptr(fused), _ptr(prior),
                                      _ptr(idx), _ptr(count), _ptr(ws), ws.numel(),
                                      _stream(stream)))
+
+
+def cc_topk_select_static(ctx: Context, desc: Desc, fused, prior, idx, count, stream=None):
+    """cc_topk_select without a workspace: for callers that cannot allocate device memory when
+    they need a selection.  The kernel's flag scratch is a fixed array inside the library
+    (CC_STATIC_SELECT_MAX_ITEMS bytes per GPU, shared by every call, so overlapping calls must
+    be ordered by the caller); larger batches raise CodecompError(CC_ERR_UNSUPPORTED).  The
+    first call on a device resolves the array's address and belongs outside stream capture."""
+    ctx.check(ctx.lib.cc_topk_select_static(ctx.handle, C.byref(desc.c), _ptr(fused), _ptr(prior),
+                                            _ptr(idx), _ptr(count), _stream(stream)))
 
 
 def cc_compact_kv(ctx: Context, desc: Desc, k, v, idx, k_out, v_out, free_pages=None,

@@ -349,6 +349,27 @@ int cc_topk_select(cc_ctx* ctx, const cc_layer_desc* desc, const float* fused, c
   return run_select(ctx, desc, p, fused, prior, idx, count, (char*)ws, stream);
 }
 
+int cc_topk_select_static(cc_ctx* ctx, const cc_layer_desc* desc, const float* fused,
+                          const float* prior, int32_t* idx, int32_t* count, void* stream) {
+  Plan p;
+  int rc = build_plan(ctx, desc, &p);
+  if (rc != CC_OK) return rc;
+  if (!fused || !prior || !count || (!idx && p.bt.b_tot > 0))
+    return fail(ctx, CC_ERR_INVALID_ARG, "NULL tensor pointer");
+  const long long need = (long long)p.g.hkv * (long long)p.bt.m_tot;
+  if (need > (long long)select_static_capacity())
+    return fail(ctx, CC_ERR_UNSUPPORTED,
+                "cc_topk_select_static: %lld flag bytes needed, the static scratch holds %lld",
+                need, (long long)select_static_capacity());
+  cudaError_t e = launch_select_static(make_launch(ctx, stream), p.bt, p.g, desc->force_threshold,
+                                       fused, prior, idx, count, ctx->device);
+  if (e == cudaErrorInvalidDevice)
+    return fail(ctx, CC_ERR_INVALID_ARG,
+                "cc_topk_select_static: the context's device must be the current device");
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "static-scratch select launch");
+  return CC_OK;
+}
+
 int cc_compact_kv(cc_ctx* ctx, const cc_layer_desc* desc, const void* k, const void* v,
                   const int32_t* idx, void* k_out, void* v_out, const int32_t* free_pages,
                   int32_t* out_page_table, void* stream) {

@@ -95,6 +95,12 @@ cudaError_t launch_select(const Launch& L, const BatchTable& bt, const Geometry&
                           float force_threshold, const float* fused, const float* prior,
                           int32_t* idx, int32_t* count, void* ws);
 
+// variant of launch_select whose scratch is a static device array (no workspace argument)
+int64_t select_static_capacity();
+cudaError_t launch_select_static(const Launch& L, const BatchTable& bt, const Geometry& g,
+                                 float force_threshold, const float* fused, const float* prior,
+                                 int32_t* idx, int32_t* count, int device);
+
 cudaError_t launch_compact(const Launch& L, const BatchTable& bt, const Geometry& g,
                            const void* k, const void* v, const int32_t* idx, void* k_out,
                            void* v_out, const int32_t* free_pages, int32_t* out_page_table);

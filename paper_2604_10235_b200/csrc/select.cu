@@ -273,7 +273,38 @@ select_kernel(const __grid_constant__ BatchTable bt, int hkv, float theta,
   if (threadIdx.x == 0) count[s * hkv + h] = (int)keep;
 }
 
+// Scratch for cc_topk_select_static: one flag byte per (head, item), resident in every GPU
+// that loads the library until the process exits.  Shared by all calls; the kernel writes
+// each flag before it reads it, so stale contents of an earlier call do no harm.
+static __device__ __align__(256) uint8_t g_static_select_flags[CC_STATIC_SELECT_MAX_ITEMS];
+
 }  // namespace
+
+int64_t select_static_capacity() { return (int64_t)CC_STATIC_SELECT_MAX_ITEMS; }
+
+cudaError_t launch_select_static(const Launch& L, const BatchTable& bt, const Geometry& g,
+                                 float force_threshold, const float* fused, const float* prior,
+                                 int32_t* idx, int32_t* count, int device) {
+  // In host code the array's name is only a handle; its device address is looked up once per
+  // device (with that device current) and cached.
+  static uint8_t* cached[64] = {nullptr};
+  if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
+  uint8_t* ptr = cached[device];
+  if (ptr == nullptr) {
+    int cur = -1;
+    cudaError_t e = cudaGetDevice(&cur);
+    if (e != cudaSuccess) return e;
+    if (cur != device) return cudaErrorInvalidDevice;
+    e = cudaGetSymbolAddress((void**)&ptr, g_static_select_flags);
+    if (e != cudaSuccess) return e;
+    if (ptr == nullptr) return cudaErrorInvalidSymbol;
+    cached[device] = ptr;
+  }
+  dim3 grid(g.hkv, bt.num_seqs);
+  select_kernel<<<grid, kThreads, 0, L.stream>>>(bt, g.hkv, force_threshold, fused, prior, idx,
+                                                 count, ptr);
+  return cudaGetLastError();
+}
 
 size_t select_ws_bytes(const BatchTable& bt, const Geometry& g) {
   return (((size_t)g.hkv * (size_t)bt.m_tot) + 255) / 256 * 256;
