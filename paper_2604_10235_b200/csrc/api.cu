@@ -207,9 +207,27 @@ int run_fuse(cc_ctx* ctx, const cc_layer_desc* d, const Plan& p, const float* sc
 
 int run_select(cc_ctx* ctx, const cc_layer_desc* d, const Plan& p, const float* fused,
                const float* prior, int32_t* idx, int32_t* count, char* ws, void* stream) {
-  cudaError_t e = launch_select(make_launch(ctx, stream), p.bt, p.g, d->force_threshold, fused,
-                                prior, idx, count, ws + p.off_select_ws);
+  const int cluster = select_cluster_size(p.bt);
+  cudaError_t e;
+  if (cluster > 0)
+    e = launch_select_cluster(make_launch(ctx, stream), p.bt, p.g, d->force_threshold, false,
+                              d->pool_kind, d->pool_size, d->alpha, d->beta, nullptr,
+                              const_cast<float*>(fused), prior, idx, count, cluster);
+  else
+    e = launch_select(make_launch(ctx, stream), p.bt, p.g, d->force_threshold, fused, prior, idx,
+                      count, ws + p.off_select_ws);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "select launch");
+  return CC_OK;
+}
+
+// pooling + prior fusion + selection in one launch (items of every sequence fit a cluster)
+int run_fuse_select(cc_ctx* ctx, const cc_layer_desc* d, const Plan& p, int cluster,
+                    const float* scores, const float* prior, float* fused, int32_t* idx,
+                    int32_t* count, void* stream) {
+  cudaError_t e = launch_select_cluster(make_launch(ctx, stream), p.bt, p.g, d->force_threshold,
+                                        true, d->pool_kind, d->pool_size, d->alpha, d->beta,
+                                        scores, fused, prior, idx, count, cluster);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "fuse + select launch");
   return CC_OK;
 }
 
@@ -400,8 +418,14 @@ int cc_compress_layer(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win,
   float* scores = (float*)(w + p.off_scores);
   float* fused = (float*)(w + p.off_fused);
   if ((rc = run_score(ctx, desc, p, q_win, k, scores, nullptr, w, stream)) != CC_OK) return rc;
-  if ((rc = run_fuse(ctx, desc, p, scores, prior, fused, stream)) != CC_OK) return rc;
-  if ((rc = run_select(ctx, desc, p, fused, prior, idx, count, w, stream)) != CC_OK) return rc;
+  const int cluster = select_cluster_size(p.bt);
+  if (cluster > 0) {
+    rc = run_fuse_select(ctx, desc, p, cluster, scores, prior, fused, idx, count, stream);
+    if (rc != CC_OK) return rc;
+  } else {
+    if ((rc = run_fuse(ctx, desc, p, scores, prior, fused, stream)) != CC_OK) return rc;
+    if ((rc = run_select(ctx, desc, p, fused, prior, idx, count, w, stream)) != CC_OK) return rc;
+  }
   if (p.bt.b_tot == 0) return CC_OK;
   return run_compact(ctx, desc, p, k, v, idx, k_out, v_out, free_pages, out_page_table, stream);
 }

@@ -95,6 +95,16 @@ cudaError_t launch_select(const Launch& L, const BatchTable& bt, const Geometry&
                           float force_threshold, const float* fused, const float* prior,
                           int32_t* idx, int32_t* count, void* ws);
 
+// cluster kernel: items resident in shared memory, optionally starting from the raw scores
+// (pooling and prior fusion done in the same launch).  select_cluster_size returns the CTAs per
+// (sequence, head) to use, or 0 when a sequence has too many items for it.
+int select_cluster_size(const BatchTable& bt);
+cudaError_t launch_select_cluster(const Launch& L, const BatchTable& bt, const Geometry& g,
+                                  float force_threshold, bool fused_input, int pool_kind,
+                                  int pool_size, float alpha, float beta, const float* scores,
+                                  float* fused, const float* prior, int32_t* idx, int32_t* count,
+                                  int cluster);
+
 // variant of launch_select whose scratch is a static device array (no workspace argument)
 int64_t select_static_capacity();
 cudaError_t launch_select_static(const Launch& L, const BatchTable& bt, const Geometry& g,

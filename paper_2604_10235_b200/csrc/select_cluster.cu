@@ -1,0 +1,498 @@
+// A2 + A3 + A4 on a thread-block cluster: pooling, prior fusion and selection of the retained
+// tokens of one (sequence, KV head) by up to eight CTAs that keep their slice of the items in
+// shared memory.
+//
+// Ranking (protected first in sequence order, then larger fused value, then lower index) and the
+// output (ascending token indices) are those of select.cu; what differs is where the data
+// lives and how the CTAs cooperate:
+//   * every item is read from global memory once; its order-preserving integer key and its
+//     protected flag stay in shared memory, so the radix descent and the ordered emission never
+//     go back to L2;
+//   * cluster-wide sums, min/max and histograms are exchanged through distributed shared
+//     memory: a CTA publishes into its own buffer, one cluster barrier later every CTA reads all
+//     peers.  Buffers alternate between two copies, which makes one barrier per exchange enough;
+//   * the cut-off is found by an 11/11/10-bit radix descent over keys shifted to the range that
+//     is present, and stops early once a bin has to be taken whole;
+//   * with FUSED the kernel starts from the raw scores: it pools them (max / avg, or sums them
+//     over a chunk), fuses them with the prior using the same explicitly rounded f32 operations
+//     as fuse_pool.cu, and also stores the fused values.
+#include <cooperative_groups.h>
+#include <string.h>
+
+#include "cc_internal.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace cc {
+
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kWarps = kThreads / 32;
+constexpr int kDigitBits = 11;
+constexpr int kBins = 1 << kDigitBits;
+constexpr int kCopies = 2;
+constexpr int kMaxCluster = 8;
+constexpr int kCtaItems = 16384;          // items one CTA keeps in shared memory
+
+struct Shared {
+  unsigned hist[2][kCopies][kBins];
+  unsigned xchg[2][4];
+  unsigned warp_a[kWarps];
+  unsigned warp_b[kWarps];
+  unsigned bcast[4];
+};
+
+struct ClusterParams {
+  int cluster;               // CTAs per (sequence, head)
+  int hkv;
+  float theta;
+  // FUSED only
+  int pool_kind, pool_size;
+  float alpha, beta;
+  const float* scores;
+  float* fused_out;
+  // plain
+  const float* fused_in;
+  const float* prior;
+  int32_t* idx;
+  int32_t* count;
+};
+
+__device__ __forceinline__ unsigned mono_key(float x) {
+  unsigned b = __float_as_uint(__fadd_rn(x, 0.0f));
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__host__ __device__ __forceinline__ int padded(int li) { return li + (li >> 5); }
+
+__device__ __forceinline__ unsigned warp_sum(unsigned v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+struct Ctx {
+  Shared* sm;
+  int C, rank;
+  unsigned phase;          // number of exchanges done so far (selects the buffer copy)
+
+  __device__ void sync_all() {
+    if (C > 1) cg::this_cluster().sync(); else __syncthreads();
+  }
+  __device__ unsigned peer(const unsigned* p, int r) const {
+    if (C == 1) return *p;
+    return *cg::this_cluster().map_shared_rank(const_cast<unsigned*>(p), r);
+  }
+
+  // sum over the block; every thread gets the result
+  __device__ unsigned block_sum(unsigned v) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) sm->warp_a[warp] = v;
+    __syncthreads();
+    return warp_sum(sm->warp_a[lane]);
+  }
+  // sum over all threads of the cluster
+  __device__ unsigned cluster_sum(unsigned v) {
+    v = block_sum(v);
+    if (C == 1) return v;
+    const unsigned b = phase++ & 1u;
+    if (threadIdx.x == 0) sm->xchg[b][0] = v;
+    sync_all();
+    unsigned t = 0;
+    for (int r = 0; r < C; ++r) t += peer(&sm->xchg[b][0], r);
+    return t;
+  }
+  __device__ void cluster_minmax(unsigned& lo, unsigned& hi) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    __syncthreads();
+    if (lane == 0) { sm->warp_a[warp] = lo; sm->warp_b[warp] = hi; }
+    __syncthreads();
+    lo = sm->warp_a[lane];
+    hi = sm->warp_b[lane];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if (C == 1) return;
+    const unsigned b = phase++ & 1u;
+    if (threadIdx.x == 0) { sm->xchg[b][0] = lo; sm->xchg[b][1] = hi; }
+    sync_all();
+    for (int r = 0; r < C; ++r) {
+      lo = min(lo, peer(&sm->xchg[b][0], r));
+      hi = max(hi, peer(&sm->xchg[b][1], r));
+    }
+  }
+  // exclusive prefix sums over the threads of the block for two counters; tot_* = block totals
+  __device__ void block_scan2(unsigned a, unsigned b, unsigned& ea, unsigned& eb,
+                              unsigned& tot_a, unsigned& tot_b) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned ia = a, ib = b;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      unsigned ta = __shfl_up_sync(0xffffffffu, ia, o);
+      unsigned tb = __shfl_up_sync(0xffffffffu, ib, o);
+      if (lane >= o) { ia += ta; ib += tb; }
+    }
+    __syncthreads();
+    if (lane == 31) { sm->warp_a[warp] = ia; sm->warp_b[warp] = ib; }
+    __syncthreads();
+    const unsigned wa = sm->warp_a[lane], wb = sm->warp_b[lane];
+    unsigned xa = wa, xb = wb;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      unsigned ta = __shfl_up_sync(0xffffffffu, xa, o);
+      unsigned tb = __shfl_up_sync(0xffffffffu, xb, o);
+      if (lane >= o) { xa += ta; xb += tb; }
+    }
+    tot_a = __shfl_sync(0xffffffffu, xa, 31);
+    tot_b = __shfl_sync(0xffffffffu, xb, 31);
+    ea = __shfl_sync(0xffffffffu, xa - wa, warp) + ia - a;
+    eb = __shfl_sync(0xffffffffu, xb - wb, warp) + ib - b;
+  }
+  // the same over all threads of the cluster (CTA rank major)
+  __device__ void cluster_scan2(unsigned a, unsigned b, unsigned& ea, unsigned& eb) {
+    unsigned ta, tb;
+    block_scan2(a, b, ea, eb, ta, tb);
+    if (C == 1) return;
+    const unsigned bf = phase++ & 1u;
+    if (threadIdx.x == 0) { sm->xchg[bf][0] = ta; sm->xchg[bf][1] = tb; }
+    sync_all();
+    for (int r = 0; r < rank; ++r) {
+      ea += peer(&sm->xchg[bf][0], r);
+      eb += peer(&sm->xchg[bf][1], r);
+    }
+  }
+};
+
+// Finds T over the eligible items such that weight(key > T) < R <= weight(key >= T), with
+// 1 <= R <= total eligible weight.  get(li, key, len) tells whether local item li is
+// eligible.  When `whole_bin` comes back true the descent stopped early: every eligible item
+// with key >= T is taken and nothing is tied.  w_above = weight strictly above the ties.
+template <class Get>
+__device__ void radix_threshold(Ctx& c, int lo, int hi, unsigned R, bool allow_early, Get get,
+                                unsigned& T, unsigned& w_above, bool& whole_bin) {
+  Shared& sm = *c.sm;
+  unsigned kmin = 0xffffffffu, kmax = 0u;
+  for (int li = lo; li < hi; ++li) {
+    unsigned key, len;
+    if (get(li, key, len)) { kmin = min(kmin, key); kmax = max(kmax, key); }
+  }
+  c.cluster_minmax(kmin, kmax);
+  const unsigned range = kmax - kmin;
+  const int sh = range ? __clz(range) : 0;
+  unsigned prefix = 0, remaining = R;
+  whole_bin = false;
+  const int copy = (threadIdx.x >> 5) & (kCopies - 1);
+  int shift = 32;
+  while (shift > 0 && range) {
+    const int bits = min(kDigitBits, shift);
+    const int hi_shift = shift;             // bits [31, hi_shift) are resolved
+    shift -= bits;
+    const unsigned b = c.phase++ & 1u;
+    unsigned* h = &sm.hist[b][0][0];
+    for (int i = threadIdx.x; i < kCopies * kBins; i += kThreads) h[i] = 0;
+    __syncthreads();
+    for (int li = lo; li < hi; ++li) {
+      unsigned key, len;
+      if (!get(li, key, len)) continue;
+      const unsigned kk = (key - kmin) << sh;
+      const bool match = hi_shift == 32 || (kk >> hi_shift) == (prefix >> hi_shift);
+      if (match) atomicAdd(&sm.hist[b][copy][(kk >> shift) & ((1u << bits) - 1u)], len);
+    }
+    c.sync_all();
+    // thread t owns bins 2047 - 2t and 2046 - 2t, so a forward scan walks the keys downwards
+    const int bin0 = kBins - 1 - 2 * (int)threadIdx.x, bin1 = bin0 - 1;
+    unsigned v0 = 0, v1 = 0;
+    for (int r = 0; r < c.C; ++r) {
+#pragma unroll
+      for (int cp = 0; cp < kCopies; ++cp) {
+        v0 += c.peer(&sm.hist[b][cp][bin0], r);
+        v1 += c.peer(&sm.hist[b][cp][bin1], r);
+      }
+    }
+    unsigned excl, d0, d1, d2;
+    c.block_scan2(v0 + v1, 0u, excl, d0, d1, d2);
+    if (excl < remaining && remaining <= excl + v0) {
+      sm.bcast[0] = (unsigned)bin0; sm.bcast[1] = remaining - excl; sm.bcast[2] = v0;
+    } else if (excl + v0 < remaining && remaining <= excl + v0 + v1) {
+      sm.bcast[0] = (unsigned)bin1; sm.bcast[1] = remaining - excl - v0; sm.bcast[2] = v1;
+    }
+    __syncthreads();
+    prefix |= sm.bcast[0] << shift;
+    remaining = sm.bcast[1];
+    const unsigned in_bin = sm.bcast[2];
+    __syncthreads();
+    if (allow_early && remaining == in_bin && shift > 0) {
+      whole_bin = true;
+      remaining = 0;
+      break;
+    }
+  }
+  T = kmin + (prefix >> sh);
+  w_above = R - remaining;
+  if (whole_bin) w_above = R;
+}
+
+template <bool FUSED>
+__global__ void __launch_bounds__(kThreads, 1)
+select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ ClusterParams P) {
+  extern __shared__ __align__(16) uint8_t dyn[];
+  Shared* smp = reinterpret_cast<Shared*>(dyn);
+  unsigned* keys = reinterpret_cast<unsigned*>(dyn + sizeof(Shared));
+  Ctx c;
+  c.sm = smp;
+  c.C = P.cluster;
+  c.rank = P.cluster > 1 ? (int)cg::this_cluster().block_rank() : 0;
+  c.phase = 0;
+
+  const int h = blockIdx.y, s = blockIdx.z;
+  const SeqInfo& q = bt.seq[s];
+  const int m = q.n_items, cs = bt.chunk;
+  const int per = (m + c.C * kThreads - 1) / (c.C * kThreads);       // items per thread
+  const int cta_lo = min(m, c.rank * kThreads * per);
+  const int cta_hi = min(m, cta_lo + kThreads * per);
+  const int cta_items = cta_hi - cta_lo;
+  uint8_t* flags = reinterpret_cast<uint8_t*>(keys + padded(kThreads * per) + 1);
+  const float* p = P.prior + q.tok_off;
+  int32_t* out = P.idx + (int64_t)h * bt.b_tot + q.idx_off;
+  const unsigned keep = (unsigned)q.keep;
+  const float theta = P.theta;
+
+  // contiguous local range of this thread
+  const int lo = min(cta_items, (int)threadIdx.x * per);
+  const int hi = min(cta_items, lo + per);
+
+  auto item_len = [&](int li) -> unsigned {
+    const int i = cta_lo + li;
+    return (unsigned)(min(q.n, (i + 1) * cs) - i * cs);
+  };
+  auto item_prior = [&](int li) -> float {
+    const int i = cta_lo + li;
+    float pr = p[(int64_t)i * cs];
+    const int end = min(q.n, (i + 1) * cs);
+    for (int j = i * cs + 1; j < end; ++j) pr = fmaxf(pr, p[j]);
+    return pr;
+  };
+
+  // ---- load: keys and protected flags of the CTA's slice (coalesced over the block)
+  if (FUSED) {
+    const float* u = P.scores + (int64_t)h * bt.n_tot + q.tok_off;
+    float* fo = P.fused_out + (int64_t)h * bt.m_tot + q.item_off;
+    const int half = (cs == 1 && P.pool_kind != CC_POOL_NONE) ? P.pool_size / 2 : 0;
+    float* us = reinterpret_cast<float*>(flags + ((kThreads * per + 15) / 16) * 16);
+    if (cs == 1 && half > 0) {
+      // stage u[cta_lo - half, cta_hi + half) (zero outside the sequence)
+      const int span = cta_items + 2 * half;
+      for (int t = threadIdx.x; t < span; t += kThreads) {
+        const int j = cta_lo - half + t;
+        us[t] = (j >= 0 && j < q.n) ? u[j] : 0.0f;
+      }
+      __syncthreads();
+    }
+    for (int li = threadIdx.x; li < cta_items; li += kThreads) {
+      const int i = cta_lo + li;
+      float val, pr;
+      if (cs > 1) {
+        const int t0 = i * cs, t1 = min(q.n, t0 + cs);
+        val = u[t0];
+        pr = p[t0];
+        for (int j = t0 + 1; j < t1; ++j) {
+          val = __fadd_rn(val, u[j]);
+          pr = fmaxf(pr, p[j]);
+        }
+      } else {
+        pr = p[i];
+        if (half == 0) {
+          val = u[i];
+        } else if (P.pool_kind == CC_POOL_MAX) {
+          val = us[li + half];
+          const int a = max(0, i - half), b = min(q.n - 1, i + half);
+          for (int j = a; j <= b; ++j) val = fmaxf(val, us[j - cta_lo + half]);
+        } else {
+          val = us[li];
+          for (int d = 1; d <= 2 * half; ++d) val = __fadd_rn(val, us[li + d]);
+          val = __fdiv_rn(val, (float)P.pool_size);
+        }
+      }
+      const float f = __fadd_rn(__fadd_rn(__fmul_rn(P.alpha, val), __fmul_rn(P.beta, pr)), 0.0f);
+      fo[i] = f;
+      keys[padded(li)] = mono_key(f);
+      flags[li] = pr >= theta ? 1 : 0;
+    }
+  } else {
+    const float* f = P.fused_in + (int64_t)h * bt.m_tot + q.item_off;
+    for (int li = threadIdx.x; li < cta_items; li += kThreads) {
+      keys[padded(li)] = mono_key(f[cta_lo + li]);
+      flags[li] = item_prior(li) >= theta ? 1 : 0;
+    }
+  }
+  __syncthreads();
+
+  // ---- stage 0: protected weight
+  unsigned wf = 0;
+  for (int li = lo; li < hi; ++li) if (flags[li]) wf += item_len(li);
+  unsigned forced_tokens = c.cluster_sum(wf);
+
+  // ---- stage 1: cap on protected items (longest prefix by (prior desc, index asc) within B_span)
+  if (q.span_cap >= 0 && forced_tokens > (unsigned)q.span_cap) {
+    const unsigned cap = (unsigned)q.span_cap;
+    unsigned t1, above1;
+    bool whole;
+    radix_threshold(c, lo, hi, cap + 1u, false,
+                    [&](int li, unsigned& key, unsigned& len) {
+                      if (!flags[li]) return false;
+                      key = mono_key(item_prior(li));
+                      len = item_len(li);
+                      return true;
+                    }, t1, above1, whole);
+    unsigned tie_w = 0;
+    for (int li = lo; li < hi; ++li)
+      if (flags[li] && mono_key(item_prior(li)) == t1) tie_w += item_len(li);
+    unsigned tie_before, dummy;
+    c.cluster_scan2(tie_w, 0u, tie_before, dummy);
+    unsigned kept = 0;
+    for (int li = lo; li < hi; ++li) {
+      if (!flags[li]) continue;
+      const unsigned key = mono_key(item_prior(li));
+      const unsigned len = item_len(li);
+      if (key > t1) { kept += len; continue; }
+      if (key == t1) {
+        const bool fits = above1 + tie_before + len <= cap;
+        tie_before += len;
+        if (fits) { kept += len; continue; }
+      }
+      flags[li] = 0;
+    }
+    forced_tokens = c.cluster_sum(kept);
+  }
+
+  // ---- stage 2: cut-off among the unprotected items
+  bool ties_are_forced, whole_bin = false;
+  unsigned t = 0, tie_budget;
+  if (forced_tokens >= keep) {
+    ties_are_forced = true;          // protected items alone fill the budget: first B in order
+    tie_budget = keep;
+  } else {
+    ties_are_forced = false;
+    unsigned above;
+    radix_threshold(c, lo, hi, keep - forced_tokens, true,
+                    [&](int li, unsigned& key, unsigned& len) {
+                      if (flags[li]) return false;
+                      key = keys[padded(li)];
+                      len = item_len(li);
+                      return true;
+                    }, t, above, whole_bin);
+    tie_budget = keep - forced_tokens - above;
+  }
+
+  // ---- stage 3: ordered emission
+  unsigned def_w = 0, tie_w = 0;
+  for (int li = lo; li < hi; ++li) {
+    const unsigned len = item_len(li);
+    if (flags[li]) {
+      if (ties_are_forced) tie_w += len; else def_w += len;
+    } else if (!ties_are_forced) {
+      const unsigned key = keys[padded(li)];
+      if (key > t || (whole_bin && key == t)) def_w += len; else if (key == t) tie_w += len;
+    }
+  }
+  unsigned def_before, tie_before;
+  c.cluster_scan2(def_w, tie_w, def_before, tie_before);
+  for (int li = lo; li < hi; ++li) {
+    const unsigned len = item_len(li);
+    unsigned take = 0;
+    bool tie = false;
+    if (flags[li]) {
+      if (ties_are_forced) tie = true; else take = len;
+    } else if (!ties_are_forced) {
+      const unsigned key = keys[padded(li)];
+      if (key > t || (whole_bin && key == t)) take = len; else if (key == t) tie = true;
+    }
+    const unsigned pos = def_before + min(tie_before, tie_budget);
+    if (tie) {
+      take = tie_before < tie_budget ? min(len, tie_budget - tie_before) : 0u;
+      tie_before += len;
+    } else {
+      def_before += take;
+    }
+    const int tok0 = (cta_lo + li) * cs;
+    for (unsigned k = 0; k < take; ++k)
+      if (pos + k < keep) out[pos + k] = tok0 + (int)k;
+  }
+  for (int i = (int)keep + c.rank * kThreads + threadIdx.x; i < q.budget; i += c.C * kThreads)
+    out[i] = -1;
+  if (c.rank == 0 && threadIdx.x == 0) P.count[s * P.hkv + h] = (int)keep;
+  // no CTA may leave while a peer can still read its shared memory
+  if (c.C > 1) cg::this_cluster().sync();
+}
+
+size_t cluster_smem_bytes(int per, bool fused, int pool_size) {
+  size_t b = sizeof(Shared);
+  b += ((size_t)padded(kThreads * per) + 1) * 4;          // keys
+  b += ((size_t)kThreads * per + 15) / 16 * 16;           // flags
+  if (fused) b += ((size_t)kThreads * per + 2 * (pool_size / 2) + 4) * 4;
+  return (b + 15) / 16 * 16;
+}
+
+}  // namespace
+
+// CTAs per (sequence, head) for the cluster kernel, or 0 when the batch does not fit.
+int select_cluster_size(const BatchTable& bt) {
+  if (bt.max_items <= 0) return 1;
+  const int target_per = 8;                       // items per thread to aim for
+  int c = 1;
+  while (c < kMaxCluster && (bt.max_items + c * kThreads - 1) / (c * kThreads) > target_per) c *= 2;
+  const int per = (bt.max_items + c * kThreads - 1) / (c * kThreads);
+  if (kThreads * per > kCtaItems) return 0;
+  return c;
+}
+
+cudaError_t launch_select_cluster(const Launch& L, const BatchTable& bt, const Geometry& g,
+                                  float force_threshold, bool fused_input, int pool_kind,
+                                  int pool_size, float alpha, float beta, const float* scores,
+                                  float* fused, const float* prior, int32_t* idx, int32_t* count,
+                                  int cluster) {
+  ClusterParams P;
+  P.cluster = cluster;
+  P.hkv = g.hkv;
+  P.theta = force_threshold;
+  P.pool_kind = pool_kind;
+  P.pool_size = pool_kind == CC_POOL_NONE ? 1 : pool_size;
+  P.alpha = alpha;
+  P.beta = beta;
+  P.scores = scores;
+  P.fused_out = fused;
+  P.fused_in = fused;
+  P.prior = prior;
+  P.idx = idx;
+  P.count = count;
+  const int per = bt.max_items > 0 ? (bt.max_items + cluster * kThreads - 1) / (cluster * kThreads) : 1;
+  const size_t smem = cluster_smem_bytes(per, fused_input, P.pool_size);
+  auto kern = fused_input ? select_cluster_kernel<true> : select_cluster_kernel<false>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(cluster, g.hkv, bt.num_seqs);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = L.stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, bt, P);
+}
+
+}  // namespace cc
