@@ -13,10 +13,22 @@
 //
 // Pipeline per CTA (one CTA per SM, 320 threads): warp 0 issues TMA loads (K tiles of 128 keys
 // through a ring of shared-memory stages, Q once per (sequence, head)), warp 1 issues
-// tcgen05.mma into two TMEM accumulator buffers, warps 2-9 drain the accumulators with
-// tcgen05.ld and do the exp / reduction work while the next tile is being multiplied.
+// tcgen05.mma into four TMEM accumulator buffers, warps 2-9 drain the accumulators with
+// tcgen05.ld and do the exp / reduction work while later tiles are being multiplied.
 // All operands sit in shared memory in the 128-byte-swizzled K-major layout that both TMA
 // and the MMA descriptors understand; Q and K simply swap the A / B roles between passes.
+//
+// TMEM holds four accumulator buffers of 128 columns; work item i (one 128 x 128 block of S or
+// S^T) lands in buffer i mod 4.  The eight epilogue warps form two sets of four (one warp per
+// TMEM lane quadrant, hence one warp of each set per scheduler); items go to the sets in pairs
+// (0, 1 -> set 0; 2, 3 -> set 1; ...).  A thread copies all 128 columns of its lane into
+// registers, hands the buffer back at once, and only then does the arithmetic, so the tensor
+// core refills buffers while the exponentials are being taken.  The exponentials are the
+// bottleneck of both passes (16 per clock on the special-function unit against 8192 tensor
+// flops per clock), so the arithmetic is written for throughput: scaling and accumulation use
+// packed f32x2 instructions, and every second pair of exponentials is evaluated on the FMA
+// pipe (round to nearest integer, degree-3 polynomial for the fraction, exponent patched in by
+// integer arithmetic; relative error 8e-5) while the other pair goes to ex2.approx.
 //
 // Every wait on an mbarrier is bounded: when the bound is hit the kernel records
 // CC_ERR_TIMEOUT, every role leaves its loop, TMEM is released and the kernel returns.
@@ -35,8 +47,10 @@ constexpr int kMaxStages = 6;
 constexpr uint32_t kPanelBytes = kTileKeys * 128;        // one 64-channel half of a K tile
 constexpr uint32_t kStageBytes = 2 * kPanelBytes;        // 32 KB
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kBufCols = 256;                        // accumulator buffer stride
-constexpr uint32_t kMiscBytes = 8192;
+constexpr uint32_t kBufCols = 128;                        // accumulator buffer stride
+constexpr int kBufs = 4;                                  // accumulator buffers in TMEM
+constexpr int kSets = 2;                                  // epilogue warp sets, two buffers each
+constexpr uint32_t kMiscBytes = 16384;
 constexpr uint32_t kSmemLimit = 232448;                   // 227 KB
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -49,7 +63,7 @@ struct TcParams {
   int w_pad;
   int n_stages;
   int n_sub;           // pass 1: 128-row blocks; pass 2: column chunks
-  int sub_cols;        // pass 2: rows per column chunk (multiple of 16, <= 256)
+  int sub_cols;        // pass 2: rows per column chunk (multiple of 16, <= 128)
   float2* part;        // [(grid + problems)][rows_pad] (max, sum) in the log2 domain
   float* scores;
   float* lse;
@@ -70,13 +84,16 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// One probe of the barrier phase; the hardware may park the thread for up to the given number
+// of nanoseconds while the phase is incomplete, so a waiting warp does not take issue slots
+// from the warps that have work.
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(2000u) : "memory");
   return ok;
 }
 __device__ __forceinline__ void fence_barrier_init() {
@@ -136,13 +153,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
         "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
       : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[8]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
-        "=r"(v[7])
-      : "r"(taddr) : "memory");
-}
 __device__ __forceinline__ void tmem_wait_ld() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
@@ -153,6 +163,100 @@ __device__ __forceinline__ float ex2(float x) {
 }
 __device__ __forceinline__ void epi_barrier() {      // the eight epilogue warps only
   asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+}
+// packed f32x2 arithmetic (two values in a 64-bit register pair per instruction)
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// 2^x for a pair on the special-function unit
+__device__ __forceinline__ uint64_t ex2_pair_sfu(uint64_t x) {
+  float a, b;
+  unpack2(x, a, b);
+  return pack2(ex2(a), ex2(b));
+}
+// 2^x for a pair on the FMA pipe: x = n + f with n = round(x) taken from the low mantissa bits
+// of x + 1.5 * 2^23, 2^f by a degree-3 minimax polynomial on [-0.5, 0.5] (relative error
+// 7.8e-5), and n added into the exponent field.  Arguments are clamped at -125 so that the
+// exponent never wraps (2^-125 is far below anything a score can resolve).
+__device__ __forceinline__ uint64_t ex2_pair_fma(uint64_t x) {
+  float a, b;
+  unpack2(x, a, b);
+  x = pack2(fmaxf(a, -125.0f), fmaxf(b, -125.0f));
+  const uint64_t magic = pack2(12582912.0f, 12582912.0f);
+  const uint64_t t = add2(x, magic);
+  const uint64_t f = sub2(x, sub2(t, magic));
+  uint64_t p = fma2(f, pack2(0.05516434833407402f, 0.05516434833407402f),
+                    pack2(0.24259322881698608f, 0.24259322881698608f));
+  p = fma2(p, f, pack2(0.693260669708252f, 0.693260669708252f));
+  p = fma2(p, f, pack2(0.9999293088912964f, 0.9999293088912964f));
+  float p0, p1, t0, t1;
+  unpack2(p, p0, p1);
+  unpack2(t, t0, t1);
+  // p * 2^n: n (low mantissa bits of t) shifted into the exponent field by one multiply-add
+  int r0, r1;
+  asm("mad.lo.s32 %0, %1, 8388608, %2;" : "=r"(r0) : "r"(__float_as_int(t0)), "r"(__float_as_int(p0)));
+  asm("mad.lo.s32 %0, %1, 8388608, %2;" : "=r"(r1) : "r"(__float_as_int(t1)), "r"(__float_as_int(p1)));
+  return pack2(__int_as_float(r0), __int_as_float(r1));
+}
+// acc += 2^(v * c + off) over the first kWidth of 32 columns; off is one pair for all columns (pass 1: -m of the
+// thread's row) or read per column from shared memory (pass 2: -L_r).
+template <bool kPerColumn, int kWidth>
+__device__ __forceinline__ void exp_accumulate(const uint32_t (&v)[32], uint64_t c2, uint64_t off2,
+                                               const float* off_col, uint64_t (&acc)[4]) {
+#pragma unroll
+  for (int i = 0; i < kWidth; i += 4) {
+    uint64_t o0 = off2, o1 = off2;
+    if (kPerColumn) {
+      const float4 L = *reinterpret_cast<const float4*>(off_col + i);
+      o0 = pack2(L.x, L.y);
+      o1 = pack2(L.z, L.w);
+    }
+    const uint64_t x0 = fma2(pack2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), c2, o0);
+    const uint64_t x1 = fma2(pack2(__uint_as_float(v[i + 2]), __uint_as_float(v[i + 3])), c2, o1);
+    acc[(i >> 2) & 1] = add2(acc[(i >> 2) & 1], ex2_pair_sfu(x0));
+    acc[2 + ((i >> 2) & 1)] = add2(acc[2 + ((i >> 2) & 1)], ex2_pair_fma(x1));
+  }
+}
+__device__ __forceinline__ float acc_total(const uint64_t (&acc)[4]) {
+  float a, b, c, d;
+  unpack2(add2(acc[0], acc[1]), a, b);
+  unpack2(add2(acc[2], acc[3]), c, d);
+  return (a + b) + (c + d);
+}
+__device__ __forceinline__ float max32(const uint32_t (&v)[32]) {
+  float m0 = max3(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]));
+  float m1 = max3(__uint_as_float(v[3]), __uint_as_float(v[4]), __uint_as_float(v[5]));
+#pragma unroll
+  for (int i = 6; i < 30; i += 4) {
+    m0 = max3(m0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+    m1 = max3(m1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+  }
+  return max3(max3(m0, m1, __uint_as_float(v[30])), __uint_as_float(v[31]), __uint_as_float(v[31]));
 }
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
@@ -176,12 +280,16 @@ struct Barriers {
   uint64_t full[kMaxStages];
   uint64_t empty[kMaxStages];
   uint64_t q_full, q_empty;
-  uint64_t acc_full[2], acc_empty[2];
+  uint64_t acc_full[kBufs], acc_empty[kBufs];
+  uint64_t u_full[8][4];             // pass 2: the other set's partial sums of (slot, quadrant)
 };
 
 struct Misc {                        // lives in the last kMiscBytes of dynamic shared memory
-  float neg_lc[kMaxRows];            // pass 2: -L_r in the log2 domain (+inf rows give 0)
-  float2 xchg[kMaxRows];             // pass 1: (max, sum) hand-over; pass 2: partial u (as .x)
+  float neg_lc[kMaxRows];            // pass 2: -L_r in the log2 domain (-1e4 for padded rows)
+  union {
+    float2 xchg[kSets][kMaxRows];    // (max, sum) hand-over: pass 1 per set, pass 2 while merging
+    float u_part[8][kTileKeys];      // pass 2: partial column sums, slot = tile & 7
+  };
   Barriers bar;
   uint32_t tmem_base;
   volatile int abort_flag;
@@ -199,7 +307,7 @@ __device__ __forceinline__ bool wait_bar(const Pipe& p, uint64_t* bar, uint32_t 
   for (uint32_t i = 0; i < 4000000u; ++i) {
     if (mbar_try_wait(b, parity)) return true;
     if (p.misc->abort_flag) return false;
-    if (i > 2048) __nanosleep(64);
+    if (i > 64) __nanosleep(200);
   }
   p.misc->abort_flag = 1;
   report_error(p.status, CC_ERR_TIMEOUT, where);
@@ -264,10 +372,12 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
     }
     mbar_init(smem_u32(&misc->bar.q_full), 1);
     mbar_init(smem_u32(&misc->bar.q_empty), 1);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kBufs; ++i) {
       mbar_init(smem_u32(&misc->bar.acc_full[i]), 1);
-      mbar_init(smem_u32(&misc->bar.acc_empty[i]), kEpiWarps);
+      mbar_init(smem_u32(&misc->bar.acc_empty[i]), 4);       // the four warps of a set
     }
+    for (int i = 0; i < 8; ++i)
+      for (int j = 0; j < 4; ++j) mbar_init(smem_u32(&misc->bar.u_full[i][j]), 1);
     misc->abort_flag = 0;
     fence_barrier_init();
   }
@@ -343,68 +453,102 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
     }
   } else if (warp == 1) {
     // ================================================================ MMA issuer
+    // One thread issues every tcgen05.mma of the CTA, so what it executes between two of them
+    // is the issue rate of the tensor pipe: descriptors are formed by adding small constants to
+    // a base word, the accumulate flag is a compile-time predicate, and the tile bookkeeping is
+    // a countdown instead of a cursor walk.
     if (lane == 0) {
       TileCursor cur;
       cur.locate(bt, g.hkv, t_begin);
-      int stage = 0, cur_problem = -1;
+      int left = cur.n_tiles - cur.local;          // tiles of the current (sequence, head) still to do
+      int stage = 0;
       uint32_t phase = 0, qf_phase = 0, item = 0;
-      const uint32_t q_addr = smem_u32(q_smem);
+      bool need_q = true;
+      // descriptor words: low = start address >> 4 | LBO field, high = SBO 1024 B, version 1,
+      // 128-byte swizzle
+      const uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+      const uint32_t q_lo0 = ((smem_u32(q_smem) & 0x3FFFFu) >> 4) | (1u << 16);
+      const uint32_t k_lo0 = ((smem_u32(k_smem) & 0x3FFFFu) >> 4) | (1u << 16);
+      const uint32_t q_panel16 = q_panel >> 4;
+      const uint32_t q_step16 = PASS == 1 ? (128u * 128u) >> 4 : ((uint32_t)P.sub_cols * 128u) >> 4;
+      const uint32_t idesc_full =
+          PASS == 1 ? instr_desc(128, kTileKeys) : instr_desc(128, (uint32_t)P.sub_cols);
+      const uint32_t idesc_last =
+          PASS == 1 ? idesc_full
+                    : instr_desc(128, (uint32_t)(P.rows_pad - (P.n_sub - 1) * P.sub_cols));
+      const uint32_t full0 = smem_u32(&misc->bar.full[0]), empty0 = smem_u32(&misc->bar.empty[0]);
+      const uint32_t accf0 = smem_u32(&misc->bar.acc_full[0]);
+      const uint32_t acce0 = smem_u32(&misc->bar.acc_empty[0]);
       bool ok = true;
       for (int t = t_begin; t < t_end && ok; ++t) {
-        if (cur.problem(g.hkv) != cur_problem) {
-          cur_problem = cur.problem(g.hkv);
+        if (need_q) {
           if (!wait_bar(pipe, &misc->bar.q_full, qf_phase, 20)) break;
           qf_phase ^= 1;
+          need_q = false;
         }
-        if (!wait_bar(pipe, &misc->bar.full[stage], phase, 21)) break;
+        if (!mbar_try_wait(full0 + 8u * (uint32_t)stage, phase) &&
+            !wait_bar(pipe, &misc->bar.full[stage], phase, 21))
+          break;
         tc_fence_after();
-        const uint32_t k_addr = smem_u32(k_smem) + (uint32_t)stage * kStageBytes;
+        const uint32_t k_lo = k_lo0 + (uint32_t)stage * (kStageBytes >> 4);
+#pragma unroll 1
         for (int sub = 0; sub < P.n_sub; ++sub, ++item) {
-          const uint32_t buf = item & 1u;
-          if (!wait_bar(pipe, &misc->bar.acc_empty[buf], ((item >> 1) & 1u) ^ 1u, 22)) {
+          const uint32_t buf = item & (kBufs - 1);
+          const uint32_t par = ((item >> 2) & 1u) ^ 1u;
+          if (!mbar_try_wait(acce0 + 8u * buf, par) &&
+              !wait_bar(pipe, &misc->bar.acc_empty[buf], par, 22)) {
             ok = false;
             break;
           }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + buf * kBufCols;
-          uint32_t idesc, q_off;
-          if (PASS == 1) {
-            idesc = instr_desc(128, kTileKeys);
-            q_off = (uint32_t)sub * 128u * 128u;                 // 128-row block of Q
-          } else {
-            const int c0 = sub * P.sub_cols;
-            const int nc = min(P.sub_cols, P.rows_pad - c0);
-            idesc = instr_desc(128, (uint32_t)nc);
-            q_off = (uint32_t)c0 * 128u;
-          }
+          const uint32_t idesc = sub == P.n_sub - 1 ? idesc_last : idesc_full;
+          const uint32_t q_lo = q_lo0 + (uint32_t)sub * q_step16;
 #pragma unroll
           for (int ks = 0; ks < kHeadDim / 16; ++ks) {
-            const uint32_t inner = (uint32_t)(ks & 3) * 32u;
-            const uint64_t qd = smem_desc(q_addr + (ks >> 2) * q_panel + q_off + inner);
-            const uint64_t kd = smem_desc(k_addr + (ks >> 2) * kPanelBytes + inner);
-            if (PASS == 1) umma_bf16(d_tmem, qd, kd, idesc, ks > 0);
-            else           umma_bf16(d_tmem, kd, qd, idesc, ks > 0);
+            const uint32_t ql = q_lo + (ks >= 4 ? q_panel16 : 0u) + (uint32_t)(ks & 3) * 2u;
+            const uint32_t kl = k_lo + (ks >= 4 ? (kPanelBytes >> 4) : 0u) + (uint32_t)(ks & 3) * 2u;
+            const uint32_t al = PASS == 1 ? ql : kl, bl = PASS == 1 ? kl : ql;
+            if (ks == 0) {
+              asm volatile(
+                  "{\n\t.reg .pred p;\n\t.reg .b64 a, b;\n\tsetp.ne.b32 p, 0, 0;\n\t"
+                  "mov.b64 a, {%1, %3};\n\tmov.b64 b, {%2, %3};\n\t"
+                  "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %4, p;\n\t}"
+                  ::"r"(d_tmem), "r"(al), "r"(bl), "r"(desc_hi), "r"(idesc) : "memory");
+            } else {
+              asm volatile(
+                  "{\n\t.reg .pred p;\n\t.reg .b64 a, b;\n\tsetp.eq.b32 p, 0, 0;\n\t"
+                  "mov.b64 a, {%1, %3};\n\tmov.b64 b, {%2, %3};\n\t"
+                  "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %4, p;\n\t}"
+                  ::"r"(d_tmem), "r"(al), "r"(bl), "r"(desc_hi), "r"(idesc) : "memory");
+            }
           }
-          umma_commit(smem_u32(&misc->bar.acc_full[buf]));
+          umma_commit(accf0 + 8u * buf);
         }
         if (!ok) break;
-        umma_commit(smem_u32(&misc->bar.empty[stage]));
+        umma_commit(empty0 + 8u * (uint32_t)stage);
         if (++stage == P.n_stages) { stage = 0; phase ^= 1; }
-        const int prev_problem = cur.problem(g.hkv);
-        cur.advance(bt, g.hkv);
-        if (t + 1 < t_end && cur.problem(g.hkv) != prev_problem)
+        if (--left == 0 && t + 1 < t_end) {
+          // the next tile belongs to another (sequence, head): Q may be replaced once the
+          // multiplications issued so far have read it
           umma_commit(smem_u32(&misc->bar.q_empty));
+          cur.local = cur.n_tiles - 1;
+          cur.advance(bt, g.hkv);
+          left = cur.n_tiles;
+          need_q = true;
+        }
       }
     }
   } else {
     // ================================================================ epilogue warps
     const int ew = warp - 2;                 // 0..7
     const int quad = warp & 3;               // TMEM lane quadrant this warp may read
-    const int half = ew >> 2;                // which half of the columns
+    const int set = ew >> 2;                 // consecutive warps cover the four quadrants
     const int row_in_tile = quad * 32 + lane;
-    const int etid = half * 128 + row_in_tile;            // 0..255, unique per epilogue thread
+    const int etid = ew * 32 + lane;         // 0..255, unique per epilogue thread
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const float c = kLog2e / sqrtf((float)kHeadDim);
+    const uint64_t c2 = pack2(c, c);
     TileCursor cur;
     cur.locate(bt, g.hkv, t_begin);
     int cur_problem = -1, cur_s = 0, cur_h = 0;
@@ -413,28 +557,23 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
     float run_m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
     float run_l[4] = {0.f, 0.f, 0.f, 0.f};
 
-    // pass 1: hand the two column halves' (max, sum) together and write the span's partial
+    // pass 1: merge the two sets' (max, sum) of every row and write the span's partial
     auto flush_partial = [&](int problem) {
 #pragma unroll
       for (int rb = 0; rb < 4; ++rb) {
         if (rb >= P.n_sub) break;
-        const int row = rb * 128 + row_in_tile;
-        if (half == 1) misc->xchg[row] = make_float2(run_m[rb], run_l[rb]);
-      }
-      epi_barrier();
-#pragma unroll
-      for (int rb = 0; rb < 4; ++rb) {
-        if (rb >= P.n_sub) break;
-        const int row = rb * 128 + row_in_tile;
-        if (half == 0 && row < P.rows_pad) {
-          const float2 o = misc->xchg[row];
-          const float m = fmaxf(run_m[rb], o.x);
-          float l = 0.f;
-          if (m > -INFINITY) l = run_l[rb] * ex2(run_m[rb] - m) + o.y * ex2(o.x - m);
-          P.part[(int64_t)(blockIdx.x + problem) * P.rows_pad + row] = make_float2(m, l);
-        }
+        misc->xchg[set][rb * 128 + row_in_tile] = make_float2(run_m[rb], run_l[rb]);
         run_m[rb] = -INFINITY;
         run_l[rb] = 0.f;
+      }
+      epi_barrier();
+      for (int row = etid; row < P.rows_pad; row += kEpiThreads) {
+        const float2 a = misc->xchg[0][row], b = misc->xchg[1][row];
+        const float m = fmaxf(a.x, b.x);
+        float l = 0.f;
+        if (a.y > 0.f) l += a.y * ex2(a.x - m);
+        if (b.y > 0.f) l += b.y * ex2(b.x - m);
+        P.part[(int64_t)(blockIdx.x + problem) * P.rows_pad + row] = make_float2(m, l);
       }
       epi_barrier();
     };
@@ -445,26 +584,57 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
         if (PASS == 1) {
           if (cur_problem >= 0) flush_partial(cur_problem);
         } else {
-          // merge the spans' (max, sum) of the new (sequence, head) into -L_r
+          // merge the spans' (max, sum) of the new (sequence, head) into -L_r: the spans are
+          // dealt round-robin to the threads that share a row, all loads of a thread are issued
+          // before the first use, and the threads of a row meet through shared memory
           epi_barrier();
           const int first_tile = g.hkv * sq.tile_off + cur.h * sq.n_tiles;
           const int b0 = cta_of_tile(first_tile, P), b1 = cta_of_tile(first_tile + sq.n_tiles - 1, P);
           const int problem = cur.problem(g.hkv);
-          for (int row = etid; row < P.rows_pad; row += kEpiThreads) {
-            float m = -INFINITY;
-            for (int b = b0; b <= b1; ++b)
-              m = fmaxf(m, P.part[(int64_t)(b + problem) * P.rows_pad + row].x);
-            float l = 0.f;
-            for (int b = b0; b <= b1; ++b) {
-              const float2 pr = P.part[(int64_t)(b + problem) * P.rows_pad + row];
-              if (pr.y > 0.f) l += pr.y * ex2(pr.x - m);
+          const int ways = max(1, min(4, kEpiThreads / P.rows_pad));    // threads per row
+          const int per_sweep = kEpiThreads / ways;                     // rows per sweep
+          float2* fold = &misc->xchg[0][0];          // no tile is in flight here, the union is free
+          for (int base = 0; base < P.rows_pad; base += per_sweep) {
+            const int row = base + etid % per_sweep, way = etid / per_sweep;
+            float m = -INFINITY, l = 0.f;
+            if (row < P.rows_pad) {
+              for (int b = b0 + way; b <= b1; b += 8 * ways) {
+                float2 pr[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                  const int bb = b + k * ways;
+                  pr[k] = bb <= b1 ? P.part[(int64_t)(bb + problem) * P.rows_pad + row]
+                                   : make_float2(-INFINITY, 0.f);
+                }
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                  if (pr[k].y > 0.f) {
+                    const float mn = fmaxf(m, pr[k].x);
+                    l = l * ex2(m - mn) + pr[k].y * ex2(pr[k].x - mn);
+                    m = mn;
+                  }
+                }
+              }
+              if (ways > 1) fold[etid] = make_float2(m, l);
             }
-            const float lc = m + log2f(l);
-            const int gq = row % g.group, tq = row / g.group;     // row = t * G + g
-            const bool real = tq < g.window;
-            misc->neg_lc[row] = real ? -lc : -INFINITY;
-            if (real && P.lse != nullptr && t == first_tile)
-              P.lse[((int64_t)cur.s * g.hq + cur.h * g.group + gq) * g.window + tq] = lc * kLn2;
+            if (ways > 1) epi_barrier();
+            if (row < P.rows_pad && way == 0) {
+              for (int k = 1; k < ways; ++k) {
+                const float2 o = fold[k * per_sweep + etid];
+                if (o.y > 0.f) {
+                  const float mn = fmaxf(m, o.x);
+                  l = l * ex2(m - mn) + o.y * ex2(o.x - mn);
+                  m = mn;
+                }
+              }
+              const float lc = m + log2f(l);
+              const int gq = row % g.group, tq = row / g.group;     // row = t * G + g
+              const bool real = tq < g.window;
+              misc->neg_lc[row] = real ? -lc : -1.0e4f;
+              if (real && P.lse != nullptr && t == first_tile)
+                P.lse[((int64_t)cur.s * g.hq + cur.h * g.group + gq) * g.window + tq] = lc * kLn2;
+            }
+            if (ways > 1) epi_barrier();
           }
           epi_barrier();
         }
@@ -474,107 +644,102 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
       }
       const int key0 = cur.local * kTileKeys;
       const int valid = min(kTileKeys, sq.n - key0);
+      const uint32_t item0 = item;          // first item of the tile
       float u_acc = 0.f;
 
 #pragma unroll 1
       for (int sub = 0; sub < P.n_sub; ++sub, ++item) {
-        const uint32_t buf = item & 1u;
+        if ((int)((item >> 1) & 1u) != set) continue;
+        const uint32_t buf = item & (kBufs - 1);
         if (!dead) {
-          const bool got = wait_bar(pipe, &misc->bar.acc_full[buf], (item >> 1) & 1u, 30);
+          // one lane probes; the vote doubles as the hand-over to the other lanes
+          const bool got = lane != 0 || wait_bar(pipe, &misc->bar.acc_full[buf], (item >> 2) & 1u, 30);
           dead = !__all_sync(0xffffffffu, got);
         }
         if (dead) continue;
         tc_fence_after();
+        // copy the lane's 128 columns into registers and hand the buffer back at once
+        uint32_t v0[32], v1[32], v2[32], v3[32];
         const uint32_t acc_addr = lane_addr + buf * kBufCols;
-        if (PASS == 1) {
-          // thread = query row (sub * 128 + row_in_tile); columns = keys of this half
-          const int col_lo = half * (kTileKeys / 2);
-          float m_run = -INFINITY, l_run = 0.f;
-#pragma unroll
-          for (int rb = 0; rb < 4; ++rb) if (rb == sub) { m_run = run_m[rb]; l_run = run_l[rb]; }
-#pragma unroll 1
-          for (int cc0 = 0; cc0 < kTileKeys / 2; cc0 += 32) {
-            uint32_t v[32];
-            tmem_ld32(acc_addr + (uint32_t)(col_lo + cc0), v);
-            tmem_wait_ld();
-            float mx = -INFINITY;
-            if (valid == kTileKeys) {
-#pragma unroll
-              for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
-            } else {
-#pragma unroll
-              for (int i = 0; i < 32; ++i) {
-                if (col_lo + cc0 + i >= valid) v[i] = 0xff800000u;       // -inf
-                mx = fmaxf(mx, __uint_as_float(v[i]));
-              }
-            }
-            const float m_new = fmaxf(m_run, mx * c);
-            if (m_new > -INFINITY) {
-              float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-              for (int i = 0; i < 32; i += 4) {
-                a0 += ex2(fmaf(__uint_as_float(v[i + 0]), c, -m_new));
-                a1 += ex2(fmaf(__uint_as_float(v[i + 1]), c, -m_new));
-                a2 += ex2(fmaf(__uint_as_float(v[i + 2]), c, -m_new));
-                a3 += ex2(fmaf(__uint_as_float(v[i + 3]), c, -m_new));
-              }
-              l_run = l_run * ex2(m_run - m_new) + ((a0 + a1) + (a2 + a3));
-              m_run = m_new;
-            }
-          }
-#pragma unroll
-          for (int rb = 0; rb < 4; ++rb) if (rb == sub) { run_m[rb] = m_run; run_l[rb] = l_run; }
-        } else {
-          // thread = key (key0 + row_in_tile); columns = query rows of this chunk's half
-          const int c0 = sub * P.sub_cols;
-          const int nc = min(P.sub_cols, P.rows_pad - c0);
-          const int hc = nc >> 1;                         // multiple of 8
-          const int col_lo = half * hc;
-          const float* nl = misc->neg_lc + c0 + col_lo;
-          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-          int cc0 = 0;
-#pragma unroll 1
-          for (; cc0 + 32 <= hc; cc0 += 32) {
-            uint32_t v[32];
-            tmem_ld32(acc_addr + (uint32_t)(col_lo + cc0), v);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-              const float4 L = *reinterpret_cast<const float4*>(nl + cc0 + i);
-              a0 += ex2(fmaf(__uint_as_float(v[i + 0]), c, L.x));
-              a1 += ex2(fmaf(__uint_as_float(v[i + 1]), c, L.y));
-              a2 += ex2(fmaf(__uint_as_float(v[i + 2]), c, L.z));
-              a3 += ex2(fmaf(__uint_as_float(v[i + 3]), c, L.w));
-            }
-          }
-#pragma unroll 1
-          for (; cc0 < hc; cc0 += 8) {
-            uint32_t v[8];
-            tmem_ld8(acc_addr + (uint32_t)(col_lo + cc0), v);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 8; i += 4) {
-              const float4 L = *reinterpret_cast<const float4*>(nl + cc0 + i);
-              a0 += ex2(fmaf(__uint_as_float(v[i + 0]), c, L.x));
-              a1 += ex2(fmaf(__uint_as_float(v[i + 1]), c, L.y));
-              a2 += ex2(fmaf(__uint_as_float(v[i + 2]), c, L.z));
-              a3 += ex2(fmaf(__uint_as_float(v[i + 3]), c, L.w));
-            }
-          }
-          u_acc += (a0 + a1) + (a2 + a3);
-        }
+        tmem_ld32(acc_addr, v0);
+        tmem_ld32(acc_addr + 32, v1);
+        tmem_ld32(acc_addr + 64, v2);
+        tmem_ld32(acc_addr + 96, v3);
+        tmem_wait_ld();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&misc->bar.acc_empty[buf]));
+        uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
+        if (PASS == 1) {
+          // thread = query row (sub * 128 + row_in_tile); columns = the 128 keys of the tile
+          if (valid != kTileKeys) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {                  // -1e4: its exponential underflows to 0
+              if (i >= valid) v0[i] = 0xc61c4000u;
+              if (32 + i >= valid) v1[i] = 0xc61c4000u;
+              if (64 + i >= valid) v2[i] = 0xc61c4000u;
+              if (96 + i >= valid) v3[i] = 0xc61c4000u;
+            }
+          }
+          float m_run = -INFINITY, l_run = 0.f;
+#pragma unroll
+          for (int rb = 0; rb < 4; ++rb) if (rb == sub) { m_run = run_m[rb]; l_run = run_l[rb]; }
+          // The reference of the exponentials only has to be near the row maximum, not equal to
+          // it: it is replaced when a value lies more than 2^64 above it.
+          const float mx = fmaxf(fmaxf(max32(v0), max32(v1)), fmaxf(max32(v2), max32(v3))) * c;
+          if (m_run == -INFINITY || mx > m_run + 64.0f) {
+            if (m_run > -INFINITY) l_run *= ex2(m_run - mx);
+            m_run = mx;
+          }
+          const uint64_t off2 = pack2(-m_run, -m_run);
+          exp_accumulate<false, 32>(v0, c2, off2, nullptr, acc);
+          exp_accumulate<false, 32>(v1, c2, off2, nullptr, acc);
+          exp_accumulate<false, 32>(v2, c2, off2, nullptr, acc);
+          exp_accumulate<false, 32>(v3, c2, off2, nullptr, acc);
+          l_run += acc_total(acc);
+#pragma unroll
+          for (int rb = 0; rb < 4; ++rb) if (rb == sub) { run_m[rb] = m_run; run_l[rb] = l_run; }
+        } else {
+          // thread = key (key0 + row_in_tile); columns = the query rows of this chunk
+          const int c0 = sub * P.sub_cols;
+          const int nc = min(P.sub_cols, P.rows_pad - c0);        // multiple of 16
+          const float* nl = misc->neg_lc + c0;
+          if (nc >= 32) exp_accumulate<true, 32>(v0, c2, 0ull, nl, acc);
+          else          exp_accumulate<true, 16>(v0, c2, 0ull, nl, acc);
+          if (nc >= 64) exp_accumulate<true, 32>(v1, c2, 0ull, nl + 32, acc);
+          else if (nc > 32) exp_accumulate<true, 16>(v1, c2, 0ull, nl + 32, acc);
+          if (nc >= 96) exp_accumulate<true, 32>(v2, c2, 0ull, nl + 64, acc);
+          else if (nc > 64) exp_accumulate<true, 16>(v2, c2, 0ull, nl + 64, acc);
+          if (nc >= 128) exp_accumulate<true, 32>(v3, c2, 0ull, nl + 96, acc);
+          else if (nc > 96) exp_accumulate<true, 16>(v3, c2, 0ull, nl + 96, acc);
+          u_acc += acc_total(acc);
+        }
       }
       if (PASS == 2) {
-        // the two column halves of a key meet through shared memory (double buffered by tile)
-        float* xu = reinterpret_cast<float*>(misc->xchg) + (t & 1) * kTileKeys;
-        if (half == 1) xu[row_in_tile] = u_acc;
-        epi_barrier();
-        if (!dead && half == 0 && row_in_tile < valid)
-          P.scores[(int64_t)cur_h * bt.n_tot + bt.seq[cur_s].tok_off + key0 + row_in_tile] =
-              u_acc + xu[row_in_tile];
+        // Items go to the sets in pairs, so the partial sums of a tile sit in one set or in
+        // both.  In the second case the set that drained the tile's last item stores; the other
+        // hands its sums over through shared memory.  Eight slots: a slot is written again only
+        // after the accumulator hand-shake has forced the reader past the tile it belongs to.
+        const int first_set = (int)((item0 >> 1) & 1u), last_set = (int)(((item - 1u) >> 1) & 1u);
+        const bool both = first_set != last_set || P.n_sub > 2;
+        const int slot = t & 7;
+        if (both && set != last_set) {
+          misc->u_part[slot][row_in_tile] = u_acc;
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&misc->bar.u_full[slot][quad]));
+        } else if (set == last_set) {
+          float u = u_acc;
+          if (both) {
+            if (!dead) {
+              const bool got = lane != 0 || wait_bar(pipe, &misc->bar.u_full[slot][quad],
+                                                     (uint32_t)((t - t_begin) >> 3) & 1u, 31);
+              dead = !__all_sync(0xffffffffu, got);
+            }
+            u += misc->u_part[slot][row_in_tile];
+          }
+          if (!dead && row_in_tile < valid)
+            P.scores[(int64_t)cur_h * bt.n_tot + bt.seq[cur_s].tok_off + key0 + row_in_tile] = u;
+        }
       }
     }
     if (PASS == 1 && cur_problem >= 0) flush_partial(cur_problem);
@@ -690,7 +855,7 @@ cudaError_t launch_score_tc(const Launch& L, const BatchTable& bt, const Geometr
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
 
-  P.n_sub = (P.rows_pad + 255) / 256;
+  P.n_sub = (P.rows_pad + 127) / 128;
   P.sub_cols = ((P.rows_pad + P.n_sub - 1) / P.n_sub + 15) / 16 * 16;
   score_tc_kernel<2><<<P.grid, kThreads, pl.smem_bytes, L.stream>>>(bt, g, P, q_map, k_map, L.status);
   return cudaGetLastError();

@@ -447,7 +447,7 @@ size_t cluster_smem_bytes(int per, bool fused, int pool_size) {
 // CTAs per (sequence, head) for the cluster kernel, or 0 when the batch does not fit.
 int select_cluster_size(const BatchTable& bt) {
   if (bt.max_items <= 0) return 1;
-  const int target_per = 8;                       // items per thread to aim for
+  const int target_per = 4;                       // items per thread to aim for
   int c = 1;
   while (c < kMaxCluster && (bt.max_items + c * kThreads - 1) / (c * kThreads) > target_per) c *= 2;
   const int per = (bt.max_items + c * kThreads - 1) / (c * kThreads);
