@@ -271,11 +271,13 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
   const int hi = min(cta_items, lo + per);
 
   auto item_len = [&](int li) -> unsigned {
+    if (cs == 1) return 1u;
     const int i = cta_lo + li;
     return (unsigned)(min(q.n, (i + 1) * cs) - i * cs);
   };
   auto item_prior = [&](int li) -> float {
     const int i = cta_lo + li;
+    if (cs == 1) return p[i];
     float pr = p[(int64_t)i * cs];
     const int end = min(q.n, (i + 1) * cs);
     for (int j = i * cs + 1; j < end; ++j) pr = fmaxf(pr, p[j]);
@@ -288,12 +290,25 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
     float* fo = P.fused_out + (int64_t)h * bt.m_tot + q.item_off;
     const int half = (cs == 1 && P.pool_kind != CC_POOL_NONE) ? P.pool_size / 2 : 0;
     float* us = reinterpret_cast<float*>(flags + ((kThreads * per + 15) / 16) * 16);
-    if (cs == 1 && half > 0) {
-      // stage u[cta_lo - half, cta_hi + half) (zero outside the sequence)
+    if (cs == 1) {
+      // stage u[cta_lo - half, cta_hi + half) (zero outside the sequence) and park the priors in
+      // the key slots; four loads of each are issued before the first store, so the slice
+      // costs a couple of round trips to L2 instead of one per item
       const int span = cta_items + 2 * half;
-      for (int t = threadIdx.x; t < span; t += kThreads) {
-        const int j = cta_lo - half + t;
-        us[t] = (j >= 0 && j < q.n) ? u[j] : 0.0f;
+      for (int t0 = threadIdx.x; t0 < span; t0 += 4 * kThreads) {
+        float a[4], b[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int t = t0 + k * kThreads, j = cta_lo - half + t;
+          a[k] = (t < span && j >= 0 && j < q.n) ? u[j] : 0.0f;
+          b[k] = t < cta_items ? p[cta_lo + t] : 0.0f;
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int t = t0 + k * kThreads;
+          if (t < span) us[t] = a[k];
+          if (t < cta_items) keys[padded(t)] = __float_as_uint(b[k]);
+        }
       }
       __syncthreads();
     }
@@ -309,9 +324,9 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
           pr = fmaxf(pr, p[j]);
         }
       } else {
-        pr = p[i];
+        pr = __uint_as_float(keys[padded(li)]);       // parked by this very thread
         if (half == 0) {
-          val = u[i];
+          val = us[li];
         } else if (P.pool_kind == CC_POOL_MAX) {
           val = us[li + half];
           const int a = max(0, i - half), b = min(q.n - 1, i + half);
@@ -406,6 +421,9 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
   }
   unsigned def_before, tie_before;
   c.cluster_scan2(def_w, tie_w, def_before, tie_before);
+  // last read of a peer's shared memory is done: announce it now, wait for the peers at the
+  // very end, and write the indices in between
+  if (c.C > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   for (int li = lo; li < hi; ++li) {
     const unsigned len = item_len(li);
     unsigned take = 0;
@@ -431,7 +449,7 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
     out[i] = -1;
   if (c.rank == 0 && threadIdx.x == 0) P.count[s * P.hkv + h] = (int)keep;
   // no CTA may leave while a peer can still read its shared memory
-  if (c.C > 1) cg::this_cluster().sync();
+  if (c.C > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 size_t cluster_smem_bytes(int per, bool fused, int pool_size) {
