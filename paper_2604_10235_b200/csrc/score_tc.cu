@@ -40,7 +40,8 @@ namespace cc {
 
 namespace {
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;                             // TMA, 2 MMA issuers, 8 epilogue warps
+constexpr int kMmaWarpB = 10;                             // second MMA issuer (set 1)
 constexpr int kEpiWarps = 8;
 constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kMaxStages = 6;
@@ -368,10 +369,10 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
   if (threadIdx.x == 0) {
     for (int i = 0; i < kMaxStages; ++i) {
       mbar_init(smem_u32(&misc->bar.full[i]), 1);
-      mbar_init(smem_u32(&misc->bar.empty[i]), 1);
+      mbar_init(smem_u32(&misc->bar.empty[i]), kSets);      // one arrival per MMA issuer
     }
     mbar_init(smem_u32(&misc->bar.q_full), 1);
-    mbar_init(smem_u32(&misc->bar.q_empty), 1);
+    mbar_init(smem_u32(&misc->bar.q_empty), kSets);
     for (int i = 0; i < kBufs; ++i) {
       mbar_init(smem_u32(&misc->bar.acc_full[i]), 1);
       mbar_init(smem_u32(&misc->bar.acc_empty[i]), 4);       // the four warps of a set
@@ -451,12 +452,15 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
         if (++stage == P.n_stages) { stage = 0; phase ^= 1; }
       }
     }
-  } else if (warp == 1) {
-    // ================================================================ MMA issuer
-    // One thread issues every tcgen05.mma of the CTA, so what it executes between two of them
-    // is the issue rate of the tensor pipe: descriptors are formed by adding small constants to
-    // a base word, the accumulate flag is a compile-time predicate, and the tile bookkeeping is
-    // a countdown instead of a cursor walk.
+  } else if (warp == 1 || warp == kMmaWarpB) {
+    // ================================================================ MMA issuers
+    // The serial instruction stream of the thread that issues tcgen05.mma (waits, descriptor
+    // words, eight multiplications and a commit per item) is what limits the tensor pipe, so
+    // there are two issuers, one per epilogue set, each taking the items of its set; both wait
+    // for every K tile and both hand it back.  Descriptors are formed by adding small constants
+    // to a base word, the accumulate flag is a compile-time predicate, and the tile bookkeeping
+    // is a countdown instead of a cursor walk.
+    const int my_set = warp == 1 ? 0 : 1;
     if (lane == 0) {
       TileCursor cur;
       cur.locate(bt, g.hkv, t_begin);
@@ -493,6 +497,7 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
         const uint32_t k_lo = k_lo0 + (uint32_t)stage * (kStageBytes >> 4);
 #pragma unroll 1
         for (int sub = 0; sub < P.n_sub; ++sub, ++item) {
+          if ((int)((item >> 1) & 1u) != my_set) continue;
           const uint32_t buf = item & (kBufs - 1);
           const uint32_t par = ((item >> 2) & 1u) ^ 1u;
           if (!mbar_try_wait(acce0 + 8u * buf, par) &&
