@@ -29,6 +29,8 @@ compact_kernel(const __grid_constant__ BatchTable bt, const Geometry g,
                const int32_t* __restrict__ idx, uint16_t* __restrict__ k_out,
                uint16_t* __restrict__ v_out, const int32_t* __restrict__ free_pages,
                int32_t* __restrict__ out_page_table, DeviceStatus* status) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int s = blockIdx.y;
   const SeqInfo& q = bt.seq[s];
   const int lane = threadIdx.x % kLanesPerRow;
@@ -89,10 +91,9 @@ cudaError_t launch_compact(const Launch& L, const BatchTable& bt, const Geometry
   const int cap = L.sm_count * 8;     // 8 resident blocks of 256 threads per SM
   if (blocks > cap) blocks = cap;
   dim3 grid(blocks, bt.num_seqs);
-  compact_kernel<<<grid, kThreads, 0, L.stream>>>(
-      bt, g, (const uint16_t*)k, (const uint16_t*)v, idx, (uint16_t*)k_out, (uint16_t*)v_out,
-      free_pages, out_page_table, L.status);
-  return cudaGetLastError();
+  return launch_pdl(compact_kernel, grid, dim3(kThreads), 0, L.stream, 1, bt, g, (const uint16_t*)k,
+                    (const uint16_t*)v, idx, (uint16_t*)k_out, (uint16_t*)v_out, free_pages,
+                    out_page_table, L.status);
 }
 
 }  // namespace cc

@@ -36,6 +36,10 @@
 
 #include "cc_internal.cuh"
 
+#ifndef CC_POLY_EVERY
+#define CC_POLY_EVERY 4
+#endif
+
 namespace cc {
 
 namespace {
@@ -55,6 +59,7 @@ constexpr uint32_t kMiscBytes = 16384;
 constexpr uint32_t kSmemLimit = 232448;                   // 227 KB
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
+constexpr int kPolyEvery = CC_POLY_EVERY;                 // one pair in this many takes the polynomial path
 
 struct TcParams {
   int grid;            // CTAs (same for both passes)
@@ -229,18 +234,18 @@ __device__ __forceinline__ uint64_t ex2_pair_fma(uint64_t x) {
 template <bool kPerColumn, int kWidth>
 __device__ __forceinline__ void exp_accumulate(const uint32_t (&v)[32], uint64_t c2, uint64_t off2,
                                                const float* off_col, uint64_t (&acc)[4]) {
+  // of every kPolyEvery pairs one goes to the FMA pipe, the others to the special-function unit
 #pragma unroll
-  for (int i = 0; i < kWidth; i += 4) {
-    uint64_t o0 = off2, o1 = off2;
+  for (int i = 0; i < kWidth; i += 2) {
+    uint64_t o = off2;
     if (kPerColumn) {
-      const float4 L = *reinterpret_cast<const float4*>(off_col + i);
-      o0 = pack2(L.x, L.y);
-      o1 = pack2(L.z, L.w);
+      const float2 L = *reinterpret_cast<const float2*>(off_col + i);
+      o = pack2(L.x, L.y);
     }
-    const uint64_t x0 = fma2(pack2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), c2, o0);
-    const uint64_t x1 = fma2(pack2(__uint_as_float(v[i + 2]), __uint_as_float(v[i + 3])), c2, o1);
-    acc[(i >> 2) & 1] = add2(acc[(i >> 2) & 1], ex2_pair_sfu(x0));
-    acc[2 + ((i >> 2) & 1)] = add2(acc[2 + ((i >> 2) & 1)], ex2_pair_fma(x1));
+    const uint64_t x = fma2(pack2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), c2, o);
+    const int pair = i >> 1;
+    if (pair % kPolyEvery == kPolyEvery - 1) acc[3] = add2(acc[3], ex2_pair_fma(x));
+    else acc[pair % 3] = add2(acc[pair % 3], ex2_pair_sfu(x));
   }
 }
 __device__ __forceinline__ float acc_total(const uint64_t (&acc)[4]) {
@@ -386,10 +391,12 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
     tmem_alloc(smem_u32(&misc->tmem_base), kTmemCols);
     tmem_relinquish();
   }
+  pdl_launch_dependents();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = misc->tmem_base;
+  pdl_wait();
 
   if (warp == 0) {
     // ================================================================ TMA producer
@@ -856,14 +863,14 @@ cudaError_t launch_score_tc(const Launch& L, const BatchTable& bt, const Geometr
 
   P.n_sub = (P.rows_pad + 127) / 128;
   P.sub_cols = 0;
-  score_tc_kernel<1><<<P.grid, kThreads, pl.smem_bytes, L.stream>>>(bt, g, P, q_map, k_map, L.status);
-  e = cudaGetLastError();
+  e = launch_pdl(score_tc_kernel<1>, dim3(P.grid), dim3(kThreads), pl.smem_bytes, L.stream, 1, bt, g, P,
+                 q_map, k_map, L.status);
   if (e != cudaSuccess) return e;
 
   P.n_sub = (P.rows_pad + 127) / 128;
   P.sub_cols = ((P.rows_pad + P.n_sub - 1) / P.n_sub + 15) / 16 * 16;
-  score_tc_kernel<2><<<P.grid, kThreads, pl.smem_bytes, L.stream>>>(bt, g, P, q_map, k_map, L.status);
-  return cudaGetLastError();
+  return launch_pdl(score_tc_kernel<2>, dim3(P.grid), dim3(kThreads), pl.smem_bytes, L.stream, 1, bt, g,
+                    P, q_map, k_map, L.status);
 }
 
 }  // namespace cc

@@ -253,6 +253,9 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
   c.rank = P.cluster > 1 ? (int)cg::this_cluster().block_rank() : 0;
   c.phase = 0;
 
+  pdl_launch_dependents();
+  pdl_wait();
+
   const int h = blockIdx.y, s = blockIdx.z;
   const SeqInfo& q = bt.seq[s];
   const int m = q.n_items, cs = bt.chunk;
@@ -497,20 +500,7 @@ cudaError_t launch_select_cluster(const Launch& L, const BatchTable& bt, const G
   auto kern = fused_input ? select_cluster_kernel<true> : select_cluster_kernel<false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  cudaLaunchConfig_t cfg;
-  memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3(cluster, g.hkv, bt.num_seqs);
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = L.stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = cluster;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, bt, P);
+  return launch_pdl(kern, dim3(cluster, g.hkv, bt.num_seqs), dim3(kThreads), smem, L.stream, cluster, bt, P);
 }
 
 }  // namespace cc
