@@ -11,24 +11,24 @@
 //   pass 2  S^T = K Q^T with keys on the M axis: one thread per key, the query rows along the
 //           TMEM columns, so u(j) is a plain in-thread sum and is stored coalesced.
 //
-// Pipeline per CTA (one CTA per SM, 320 threads): warp 0 issues TMA loads (K tiles of 128 keys
-// through a ring of shared-memory stages, Q once per (sequence, head)), warp 1 issues
-// tcgen05.mma into four TMEM accumulator buffers, warps 2-9 drain the accumulators with
+// Pipeline per CTA (one CTA per SM, 608 threads): warp 0 issues TMA loads (K tiles of 128 keys
+// through a ring of shared-memory stages, Q once per (sequence, head)), two warps issue
+// tcgen05.mma into four TMEM accumulator buffers, sixteen warps drain the accumulators with
 // tcgen05.ld and do the exp / reduction work while later tiles are being multiplied.
 // All operands sit in shared memory in the 128-byte-swizzled K-major layout that both TMA
 // and the MMA descriptors understand; Q and K simply swap the A / B roles between passes.
 //
 // TMEM holds four accumulator buffers of 128 columns; work item i (one 128 x 128 block of S or
-// S^T) lands in buffer i mod 4.  The eight epilogue warps form two sets of four (one warp per
-// TMEM lane quadrant, hence one warp of each set per scheduler); items go to the sets in pairs
-// (0, 1 -> set 0; 2, 3 -> set 1; ...).  A thread copies all 128 columns of its lane into
-// registers, hands the buffer back at once, and only then does the arithmetic, so the tensor
-// core refills buffers while the exponentials are being taken.  The exponentials are the
-// bottleneck of both passes (16 per clock on the special-function unit against 8192 tensor
-// flops per clock), so the arithmetic is written for throughput: scaling and accumulation use
-// packed f32x2 instructions, and every second pair of exponentials is evaluated on the FMA
-// pipe (round to nearest integer, degree-3 polynomial for the fraction, exponent patched in by
-// integer arithmetic; relative error 8e-5) while the other pair goes to ex2.approx.
+// S^T) lands in buffer i mod 4.  The sixteen epilogue warps form four sets of four (one warp
+// per TMEM lane quadrant); set k drains buffer k, so every scheduler hosts one warp of each set
+// and the sets run staggered: while one set waits for its buffer to be refilled, the other
+// three keep the special-function unit busy.  The exponentials are the bottleneck of both
+// passes (16 per clock on the special-function unit against 8192 tensor flops per clock), and
+// what counts is that the unit never idles: a warp reads 32 columns at a time, so it needs few
+// registers and four warps fit per scheduler; scaling and accumulation use packed f32x2
+// instructions; one pair of exponentials in kPolyEvery is evaluated on the FMA pipe instead
+// (round to nearest integer, degree-3 polynomial for the fraction, exponent patched in by
+// integer arithmetic; relative error 8e-5).
 //
 // Every wait on an mbarrier is bounded: when the bound is hit the kernel records
 // CC_ERR_TIMEOUT, every role leaves its loop, TMEM is released and the kernel returns.
@@ -44,9 +44,10 @@ namespace cc {
 
 namespace {
 
-constexpr int kThreads = 352;                             // TMA, 2 MMA issuers, 8 epilogue warps
-constexpr int kMmaWarpB = 10;                             // second MMA issuer (set 1)
-constexpr int kEpiWarps = 8;
+constexpr int kThreads = 608;                             // TMA, 2 MMA issuers, 16 epilogue warps
+constexpr int kMmaWarpB = 18;                             // second MMA issuer
+constexpr int kIssuers = 2;
+constexpr int kEpiWarps = 16;
 constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kMaxStages = 6;
 constexpr uint32_t kPanelBytes = kTileKeys * 128;        // one 64-channel half of a K tile
@@ -54,8 +55,8 @@ constexpr uint32_t kStageBytes = 2 * kPanelBytes;        // 32 KB
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kBufCols = 128;                        // accumulator buffer stride
 constexpr int kBufs = 4;                                  // accumulator buffers in TMEM
-constexpr int kSets = 2;                                  // epilogue warp sets, two buffers each
-constexpr uint32_t kMiscBytes = 16384;
+constexpr int kSets = 4;                                  // epilogue warp sets, one per buffer
+constexpr uint32_t kMiscBytes = 20480;
 constexpr uint32_t kSmemLimit = 232448;                   // 227 KB
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -86,6 +87,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_n(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -167,7 +171,7 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ void epi_barrier() {      // the eight epilogue warps only
+__device__ __forceinline__ void epi_barrier() {      // the sixteen epilogue warps only
   asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
 }
 // packed f32x2 arithmetic (two values in a 64-bit register pair per instruction)
@@ -287,14 +291,14 @@ struct Barriers {
   uint64_t empty[kMaxStages];
   uint64_t q_full, q_empty;
   uint64_t acc_full[kBufs], acc_empty[kBufs];
-  uint64_t u_full[8][4];             // pass 2: the other set's partial sums of (slot, quadrant)
+  uint64_t u_full[8][4];             // pass 2: the other sets' partial sums of (slot, quadrant)
 };
 
 struct Misc {                        // lives in the last kMiscBytes of dynamic shared memory
   float neg_lc[kMaxRows];            // pass 2: -L_r in the log2 domain (-1e4 for padded rows)
   union {
     float2 xchg[kSets][kMaxRows];    // (max, sum) hand-over: pass 1 per set, pass 2 while merging
-    float u_part[8][kTileKeys];      // pass 2: partial column sums, slot = tile & 7
+    float u_part[8][kSets][kTileKeys];   // pass 2: partial column sums, slot = tile & 7
   };
   Barriers bar;
   uint32_t tmem_base;
@@ -374,16 +378,16 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
   if (threadIdx.x == 0) {
     for (int i = 0; i < kMaxStages; ++i) {
       mbar_init(smem_u32(&misc->bar.full[i]), 1);
-      mbar_init(smem_u32(&misc->bar.empty[i]), kSets);      // one arrival per MMA issuer
+      mbar_init(smem_u32(&misc->bar.empty[i]), kIssuers);   // one arrival per MMA issuer
     }
     mbar_init(smem_u32(&misc->bar.q_full), 1);
-    mbar_init(smem_u32(&misc->bar.q_empty), kSets);
+    mbar_init(smem_u32(&misc->bar.q_empty), kIssuers);
     for (int i = 0; i < kBufs; ++i) {
       mbar_init(smem_u32(&misc->bar.acc_full[i]), 1);
       mbar_init(smem_u32(&misc->bar.acc_empty[i]), 4);       // the four warps of a set
     }
     for (int i = 0; i < 8; ++i)
-      for (int j = 0; j < 4; ++j) mbar_init(smem_u32(&misc->bar.u_full[i][j]), 1);
+      for (int j = 0; j < 4; ++j) mbar_init(smem_u32(&misc->bar.u_full[i][j]), kSets - 1);
     misc->abort_flag = 0;
     fence_barrier_init();
   }
@@ -461,13 +465,13 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
     }
   } else if (warp == 1 || warp == kMmaWarpB) {
     // ================================================================ MMA issuers
-    // The serial instruction stream of the thread that issues tcgen05.mma (waits, descriptor
-    // words, eight multiplications and a commit per item) is what limits the tensor pipe, so
-    // there are two issuers, one per epilogue set, each taking the items of its set; both wait
-    // for every K tile and both hand it back.  Descriptors are formed by adding small constants
+    // The serial instruction stream of a thread that issues tcgen05.mma (waits, descriptor
+    // words, eight multiplications and a commit per item) is long, so there are two issuers;
+    // items go to them in pairs (0, 1 -> first; 2, 3 -> second; ...); both wait for every K
+    // tile and both hand it back.  Descriptors are formed by adding small constants
     // to a base word, the accumulate flag is a compile-time predicate, and the tile bookkeeping
     // is a countdown instead of a cursor walk.
-    const int my_set = warp == 1 ? 0 : 1;
+    const int my_half = warp == 1 ? 0 : 1;
     if (lane == 0) {
       TileCursor cur;
       cur.locate(bt, g.hkv, t_begin);
@@ -504,7 +508,7 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
         const uint32_t k_lo = k_lo0 + (uint32_t)stage * (kStageBytes >> 4);
 #pragma unroll 1
         for (int sub = 0; sub < P.n_sub; ++sub, ++item) {
-          if ((int)((item >> 1) & 1u) != my_set) continue;
+          if ((int)((item >> 1) & 1u) != my_half) continue;
           const uint32_t buf = item & (kBufs - 1);
           const uint32_t par = ((item >> 2) & 1u) ^ 1u;
           if (!mbar_try_wait(acce0 + 8u * buf, par) &&
@@ -553,11 +557,11 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
     }
   } else {
     // ================================================================ epilogue warps
-    const int ew = warp - 2;                 // 0..7
+    const int ew = warp - 2;                 // 0..15
     const int quad = warp & 3;               // TMEM lane quadrant this warp may read
     const int set = ew >> 2;                 // consecutive warps cover the four quadrants
     const int row_in_tile = quad * 32 + lane;
-    const int etid = ew * 32 + lane;         // 0..255, unique per epilogue thread
+    const int etid = ew * 32 + lane;         // 0..511, unique per epilogue thread
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const float c = kLog2e / sqrtf((float)kHeadDim);
     const uint64_t c2 = pack2(c, c);
@@ -569,7 +573,7 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
     float run_m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
     float run_l[4] = {0.f, 0.f, 0.f, 0.f};
 
-    // pass 1: merge the two sets' (max, sum) of every row and write the span's partial
+    // pass 1: merge the four sets' (max, sum) of every row and write the span's partial
     auto flush_partial = [&](int problem) {
 #pragma unroll
       for (int rb = 0; rb < 4; ++rb) {
@@ -580,11 +584,15 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
       }
       epi_barrier();
       for (int row = etid; row < P.rows_pad; row += kEpiThreads) {
-        const float2 a = misc->xchg[0][row], b = misc->xchg[1][row];
-        const float m = fmaxf(a.x, b.x);
+        float m = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < kSets; ++k) m = fmaxf(m, misc->xchg[k][row].x);
         float l = 0.f;
-        if (a.y > 0.f) l += a.y * ex2(a.x - m);
-        if (b.y > 0.f) l += b.y * ex2(b.x - m);
+#pragma unroll
+        for (int k = 0; k < kSets; ++k) {
+          const float2 o = misc->xchg[k][row];
+          if (o.y > 0.f) l += o.y * ex2(o.x - m);
+        }
         P.part[(int64_t)(blockIdx.x + problem) * P.rows_pad + row] = make_float2(m, l);
       }
       epi_barrier();
@@ -661,8 +669,8 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
 
 #pragma unroll 1
       for (int sub = 0; sub < P.n_sub; ++sub, ++item) {
-        if ((int)((item >> 1) & 1u) != set) continue;
         const uint32_t buf = item & (kBufs - 1);
+        if ((int)buf != set) continue;
         if (!dead) {
           // one lane probes; the vote doubles as the hand-over to the other lanes
           const bool got = lane != 0 || wait_bar(pipe, &misc->bar.acc_full[buf], (item >> 2) & 1u, 30);
@@ -670,44 +678,39 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
         }
         if (dead) continue;
         tc_fence_after();
-        // copy the lane's 128 columns into registers and hand the buffer back at once
-        uint32_t v0[32], v1[32], v2[32], v3[32];
         const uint32_t acc_addr = lane_addr + buf * kBufCols;
-        tmem_ld32(acc_addr, v0);
-        tmem_ld32(acc_addr + 32, v1);
-        tmem_ld32(acc_addr + 64, v2);
-        tmem_ld32(acc_addr + 96, v3);
-        tmem_wait_ld();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&misc->bar.acc_empty[buf]));
         uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
+        uint32_t v[32];
         if (PASS == 1) {
           // thread = query row (sub * 128 + row_in_tile); columns = the 128 keys of the tile
-          if (valid != kTileKeys) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {                  // -1e4: its exponential underflows to 0
-              if (i >= valid) v0[i] = 0xc61c4000u;
-              if (32 + i >= valid) v1[i] = 0xc61c4000u;
-              if (64 + i >= valid) v2[i] = 0xc61c4000u;
-              if (96 + i >= valid) v3[i] = 0xc61c4000u;
-            }
-          }
           float m_run = -INFINITY, l_run = 0.f;
 #pragma unroll
           for (int rb = 0; rb < 4; ++rb) if (rb == sub) { m_run = run_m[rb]; l_run = run_l[rb]; }
-          // The reference of the exponentials only has to be near the row maximum, not equal to
-          // it: it is replaced when a value lies more than 2^64 above it.
-          const float mx = fmaxf(fmaxf(max32(v0), max32(v1)), fmaxf(max32(v2), max32(v3))) * c;
-          if (m_run == -INFINITY || mx > m_run + 64.0f) {
-            if (m_run > -INFINITY) l_run *= ex2(m_run - mx);
-            m_run = mx;
+#pragma unroll 1
+          for (int cc0 = 0; cc0 < kTileKeys; cc0 += 32) {
+            tmem_ld32(acc_addr + (uint32_t)cc0, v);
+            tmem_wait_ld();
+            if (cc0 + 32 == kTileKeys) {             // last read of the buffer: hand it back
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(smem_u32(&misc->bar.acc_empty[buf]));
+            }
+            if (cc0 >= valid) continue;
+            if (cc0 + 32 > valid) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (cc0 + i >= valid) v[i] = 0xc61c4000u;    // -1e4: its exponential underflows to 0
+            }
+            // The reference of the exponentials only has to be near the row maximum, not equal
+            // to it: it is replaced when a value lies more than 2^64 above it.
+            const float mx = max32(v) * c;
+            if (m_run == -INFINITY || mx > m_run + 64.0f) {
+              if (m_run > -INFINITY) l_run = (l_run + acc_total(acc)) * ex2(m_run - mx);
+              acc[0] = acc[1] = acc[2] = acc[3] = 0ull;
+              m_run = mx;
+            }
+            exp_accumulate<false, 32>(v, c2, pack2(-m_run, -m_run), nullptr, acc);
           }
-          const uint64_t off2 = pack2(-m_run, -m_run);
-          exp_accumulate<false, 32>(v0, c2, off2, nullptr, acc);
-          exp_accumulate<false, 32>(v1, c2, off2, nullptr, acc);
-          exp_accumulate<false, 32>(v2, c2, off2, nullptr, acc);
-          exp_accumulate<false, 32>(v3, c2, off2, nullptr, acc);
           l_run += acc_total(acc);
 #pragma unroll
           for (int rb = 0; rb < 4; ++rb) if (rb == sub) { run_m[rb] = m_run; run_l[rb] = l_run; }
@@ -716,42 +719,53 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
           const int c0 = sub * P.sub_cols;
           const int nc = min(P.sub_cols, P.rows_pad - c0);        // multiple of 16
           const float* nl = misc->neg_lc + c0;
-          if (nc >= 32) exp_accumulate<true, 32>(v0, c2, 0ull, nl, acc);
-          else          exp_accumulate<true, 16>(v0, c2, 0ull, nl, acc);
-          if (nc >= 64) exp_accumulate<true, 32>(v1, c2, 0ull, nl + 32, acc);
-          else if (nc > 32) exp_accumulate<true, 16>(v1, c2, 0ull, nl + 32, acc);
-          if (nc >= 96) exp_accumulate<true, 32>(v2, c2, 0ull, nl + 64, acc);
-          else if (nc > 64) exp_accumulate<true, 16>(v2, c2, 0ull, nl + 64, acc);
-          if (nc >= 128) exp_accumulate<true, 32>(v3, c2, 0ull, nl + 96, acc);
-          else if (nc > 96) exp_accumulate<true, 16>(v3, c2, 0ull, nl + 96, acc);
+#pragma unroll 1
+          for (int cc0 = 0; cc0 < nc; cc0 += 32) {
+            tmem_ld32(acc_addr + (uint32_t)cc0, v);               // stays inside the 128-column buffer
+            tmem_wait_ld();
+            if (cc0 + 32 >= nc) {
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(smem_u32(&misc->bar.acc_empty[buf]));
+            }
+            if (cc0 + 32 <= nc) exp_accumulate<true, 32>(v, c2, 0ull, nl + cc0, acc);
+            else                exp_accumulate<true, 16>(v, c2, 0ull, nl + cc0, acc);
+          }
           u_acc += acc_total(acc);
         }
       }
-      if (PASS == 2) {
-        // Items go to the sets in pairs, so the partial sums of a tile sit in one set or in
-        // both.  In the second case the set that drained the tile's last item stores; the other
-        // hands its sums over through shared memory.  Eight slots: a slot is written again only
-        // after the accumulator hand-shake has forced the reader past the tile it belongs to.
-        const int first_set = (int)((item0 >> 1) & 1u), last_set = (int)(((item - 1u) >> 1) & 1u);
-        const bool both = first_set != last_set || P.n_sub > 2;
+      if (PASS == 2 && P.n_sub > 1) {
+        // The sets that hold partial sums of the tile (one per item) meet through shared
+        // memory: the set that drained the tile's last item adds the others' sums and stores.
+        // kSets - 1 arrivals complete a (slot, quadrant); the storing warp tops up what is
+        // missing when the tile has fewer than four items.  Eight slots: a slot is written again
+        // only after the accumulator hand-shake has forced the reader past the tile it belongs to.
+        const int n_items = (int)(item - item0);                  // 2..4
+        const int last_set = (int)((item - 1u) & (kBufs - 1));
+        const bool worked = ((uint32_t)(set - (int)(item0 & (kBufs - 1))) & (kBufs - 1)) < (uint32_t)n_items;
         const int slot = t & 7;
-        if (both && set != last_set) {
-          misc->u_part[slot][row_in_tile] = u_acc;
+        if (worked && set != last_set) {
+          misc->u_part[slot][set][row_in_tile] = u_acc;
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(&misc->bar.u_full[slot][quad]));
         } else if (set == last_set) {
-          float u = u_acc;
-          if (both) {
-            if (!dead) {
-              const bool got = lane != 0 || wait_bar(pipe, &misc->bar.u_full[slot][quad],
-                                                     (uint32_t)((t - t_begin) >> 3) & 1u, 31);
-              dead = !__all_sync(0xffffffffu, got);
-            }
-            u += misc->u_part[slot][row_in_tile];
+          if (lane == 0 && n_items < kSets)
+            mbar_arrive_n(smem_u32(&misc->bar.u_full[slot][quad]), (uint32_t)(kSets - n_items));
+          if (!dead) {
+            const bool got = lane != 0 || wait_bar(pipe, &misc->bar.u_full[slot][quad],
+                                                   (uint32_t)((t - t_begin) >> 3) & 1u, 31);
+            dead = !__all_sync(0xffffffffu, got);
           }
-          if (!dead && row_in_tile < valid)
+          if (!dead && row_in_tile < valid) {
+            float u = u_acc;
+            for (int k = 1; k < n_items; ++k)
+              u += misc->u_part[slot][(last_set + kSets - k) & (kSets - 1)][row_in_tile];
             P.scores[(int64_t)cur_h * bt.n_tot + bt.seq[cur_s].tok_off + key0 + row_in_tile] = u;
+          }
         }
+      } else if (PASS == 2) {
+        if ((int)(item0 & (kBufs - 1)) == set && !dead && row_in_tile < valid)
+          P.scores[(int64_t)cur_h * bt.n_tot + bt.seq[cur_s].tok_off + key0 + row_in_tile] = u_acc;
       }
     }
     if (PASS == 1 && cur_problem >= 0) flush_partial(cur_problem);
