@@ -567,7 +567,7 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
     const uint64_t c2 = pack2(c, c);
     TileCursor cur;
     cur.locate(bt, g.hkv, t_begin);
-    int cur_problem = -1, cur_s = 0, cur_h = 0;
+    int cur_problem = -1;
     uint32_t item = 0;
     bool dead = false;      // after a failed wait: keep the loop structure (and its barriers), skip the work
     float run_m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -598,9 +598,17 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
       epi_barrier();
     };
 
-    for (int t = t_begin; t < t_end; ++t, cur.advance(bt, g.hkv)) {
-      const SeqInfo& sq = bt.seq[cur.s];
-      if (cur.problem(g.hkv) != cur_problem) {
+    // the cursor is walked only where the (sequence, head) changes; in between a countdown and
+    // a running key offset describe the tile
+    int left = 0, key0 = 0, n_cur = 0;
+    int64_t out_base = 0;
+    for (int t = t_begin; t < t_end; ++t, key0 += kTileKeys, --left) {
+      if (left == 0) {
+        if (cur_problem >= 0) {
+          cur.local = cur.n_tiles - 1;
+          cur.advance(bt, g.hkv);
+        }
+        const SeqInfo& sq = bt.seq[cur.s];
         if (PASS == 1) {
           if (cur_problem >= 0) flush_partial(cur_problem);
         } else {
@@ -659,11 +667,12 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
           epi_barrier();
         }
         cur_problem = cur.problem(g.hkv);
-        cur_s = cur.s;
-        cur_h = cur.h;
+        left = cur.n_tiles - cur.local;
+        key0 = cur.local * kTileKeys;
+        n_cur = sq.n;
+        out_base = (int64_t)cur.h * bt.n_tot + sq.tok_off;
       }
-      const int key0 = cur.local * kTileKeys;
-      const int valid = min(kTileKeys, sq.n - key0);
+      const int valid = min(kTileKeys, n_cur - key0);
       const uint32_t item0 = item;          // first item of the tile
       float u_acc = 0.f;
 
@@ -760,12 +769,12 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
             float u = u_acc;
             for (int k = 1; k < n_items; ++k)
               u += misc->u_part[slot][(last_set + kSets - k) & (kSets - 1)][row_in_tile];
-            P.scores[(int64_t)cur_h * bt.n_tot + bt.seq[cur_s].tok_off + key0 + row_in_tile] = u;
+            P.scores[out_base + key0 + row_in_tile] = u;
           }
         }
       } else if (PASS == 2) {
         if ((int)(item0 & (kBufs - 1)) == set && !dead && row_in_tile < valid)
-          P.scores[(int64_t)cur_h * bt.n_tot + bt.seq[cur_s].tok_off + key0 + row_in_tile] = u_acc;
+          P.scores[out_base + key0 + row_in_tile] = u_acc;
       }
     }
     if (PASS == 1 && cur_problem >= 0) flush_partial(cur_problem);
