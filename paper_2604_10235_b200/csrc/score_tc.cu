@@ -240,16 +240,20 @@ __device__ __forceinline__ void exp_accumulate(const uint32_t (&v)[32], uint64_t
                                                const float* off_col, uint64_t (&acc)[4]) {
   // of every kPolyEvery pairs one goes to the FMA pipe, the others to the special-function unit
 #pragma unroll
-  for (int i = 0; i < kWidth; i += 2) {
-    uint64_t o = off2;
+  for (int i = 0; i < kWidth; i += 4) {
+    uint64_t o[2] = {off2, off2};
     if (kPerColumn) {
-      const float2 L = *reinterpret_cast<const float2*>(off_col + i);
-      o = pack2(L.x, L.y);
+      const float4 L = *reinterpret_cast<const float4*>(off_col + i);
+      o[0] = pack2(L.x, L.y);
+      o[1] = pack2(L.z, L.w);
     }
-    const uint64_t x = fma2(pack2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), c2, o);
-    const int pair = i >> 1;
-    if (pair % kPolyEvery == kPolyEvery - 1) acc[3] = add2(acc[3], ex2_pair_fma(x));
-    else acc[pair % 3] = add2(acc[pair % 3], ex2_pair_sfu(x));
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int pair = (i >> 1) + k;
+      const uint64_t x = fma2(pack2(__uint_as_float(v[i + 2 * k]), __uint_as_float(v[i + 2 * k + 1])), c2, o[k]);
+      if (pair % kPolyEvery == kPolyEvery - 1) acc[3] = add2(acc[3], ex2_pair_fma(x));
+      else acc[pair % 3] = add2(acc[pair % 3], ex2_pair_sfu(x));
+    }
   }
 }
 __device__ __forceinline__ float acc_total(const uint64_t (&acc)[4]) {
