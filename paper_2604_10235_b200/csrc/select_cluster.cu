@@ -319,12 +319,24 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
       const int i = cta_lo + li;
       float val, pr;
       if (cs > 1) {
+        // chunk sum in token order; the loads of eight tokens are issued before they are used
         const int t0 = i * cs, t1 = min(q.n, t0 + cs);
-        val = u[t0];
-        pr = p[t0];
-        for (int j = t0 + 1; j < t1; ++j) {
-          val = __fadd_rn(val, u[j]);
-          pr = fmaxf(pr, p[j]);
+        val = 0.0f;
+        pr = -INFINITY;
+        for (int j0 = t0; j0 < t1; j0 += 8) {
+          float a[8], b[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            a[k] = j0 + k < t1 ? u[j0 + k] : 0.0f;
+            b[k] = j0 + k < t1 ? p[j0 + k] : -INFINITY;
+          }
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            if (j0 + k < t1) {
+              val = (j0 + k == t0) ? a[k] : __fadd_rn(val, a[k]);
+              pr = fmaxf(pr, b[k]);
+            }
+          }
         }
       } else {
         pr = __uint_as_float(keys[padded(li)]);       // parked by this very thread
@@ -470,7 +482,9 @@ int select_cluster_size(const BatchTable& bt) {
   if (bt.max_items <= 0) return 1;
   const int target_per = 4;                       // items per thread to aim for
   int c = 1;
-  while (c < kMaxCluster && (bt.max_items + c * kThreads - 1) / (c * kThreads) > target_per) c *= 2;
+  // in chunk mode a thread reads all tokens of its items, so the width is chosen by tokens
+  const long long work = (long long)bt.max_items * bt.chunk;
+  while (c < kMaxCluster && (work + c * kThreads - 1) / (c * kThreads) > target_per) c *= 2;
   const int per = (bt.max_items + c * kThreads - 1) / (c * kThreads);
   if (kThreads * per > kCtaItems) return 0;
   return c;
