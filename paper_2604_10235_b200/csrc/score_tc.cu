@@ -37,7 +37,7 @@
 #include "cc_internal.cuh"
 
 #ifndef CC_POLY_EVERY
-#define CC_POLY_EVERY 4
+#define CC_POLY_EVERY 3
 #endif
 
 namespace cc {
