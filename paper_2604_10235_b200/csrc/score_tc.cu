@@ -676,8 +676,12 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
         n_cur = sq.n;
         out_base = (int64_t)cur.h * bt.n_tot + sq.tok_off;
       }
-      const int valid = min(kTileKeys, n_cur - key0);
       const uint32_t item0 = item;          // first item of the tile
+      if (((uint32_t)(set - (int)(item0 & (kBufs - 1))) & (kBufs - 1)) >= (uint32_t)P.n_sub) {
+        item += (uint32_t)P.n_sub;          // none of the tile's items is this set's
+        continue;
+      }
+      const int valid = min(kTileKeys, n_cur - key0);
       float u_acc = 0.f;
 
 #pragma unroll 1
