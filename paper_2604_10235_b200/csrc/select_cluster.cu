@@ -11,7 +11,7 @@
 //   * cluster-wide sums, min/max and histograms are exchanged through distributed shared
 //     memory: a CTA publishes into its own buffer, one cluster barrier later every CTA reads all
 //     peers.  Buffers alternate between two copies, which makes one barrier per exchange enough;
-//   * the cut-off is found by an 11/11/10-bit radix descent over keys shifted to the range that
+//   * the cut-off is found by an four-step 8-bit radix descent over keys shifted to the range that
 //     is present, and stops early once a bin has to be taken whole;
 //   * with FUSED the kernel starts from the raw scores: it pools them (max / avg, or sums them
 //     over a chunk), fuses them with the prior using the same explicitly rounded f32 operations
@@ -29,7 +29,7 @@ namespace {
 
 constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
-constexpr int kDigitBits = 11;
+constexpr int kDigitBits = 8;
 constexpr int kBins = 1 << kDigitBits;
 constexpr int kCopies = 2;
 constexpr int kMaxCluster = 8;
@@ -207,23 +207,24 @@ __device__ void radix_threshold(Ctx& c, int lo, int hi, unsigned R, bool allow_e
       const bool match = hi_shift == 32 || (kk >> hi_shift) == (prefix >> hi_shift);
       if (match) atomicAdd(&sm.hist[b][copy][(kk >> shift) & ((1u << bits) - 1u)], len);
     }
-    c.sync_all();
-    // thread t owns bins 2047 - 2t and 2046 - 2t, so a forward scan walks the keys downwards
-    const int bin0 = kBins - 1 - 2 * (int)threadIdx.x, bin1 = bin0 - 1;
-    unsigned v0 = 0, v1 = 0;
-    for (int r = 0; r < c.C; ++r) {
+    // fold the private copies into copy 0 before the peers look at it
+    __syncthreads();
+    if (threadIdx.x < kBins) {
+      unsigned t = sm.hist[b][0][threadIdx.x];
 #pragma unroll
-      for (int cp = 0; cp < kCopies; ++cp) {
-        v0 += c.peer(&sm.hist[b][cp][bin0], r);
-        v1 += c.peer(&sm.hist[b][cp][bin1], r);
-      }
+      for (int cp = 1; cp < kCopies; ++cp) t += sm.hist[b][cp][threadIdx.x];
+      sm.hist[b][0][threadIdx.x] = t;
     }
+    c.sync_all();
+    // thread t (< 256) owns bin 255 - t, so a forward scan walks the keys downwards
+    const int bin0 = kBins - 1 - (int)threadIdx.x;
+    unsigned v0 = 0;
+    if (threadIdx.x < kBins)
+      for (int r = 0; r < c.C; ++r) v0 += c.peer(&sm.hist[b][0][bin0], r);
     unsigned excl, d0, d1, d2;
-    c.block_scan2(v0 + v1, 0u, excl, d0, d1, d2);
-    if (excl < remaining && remaining <= excl + v0) {
+    c.block_scan2(v0, 0u, excl, d0, d1, d2);
+    if (threadIdx.x < kBins && excl < remaining && remaining <= excl + v0) {
       sm.bcast[0] = (unsigned)bin0; sm.bcast[1] = remaining - excl; sm.bcast[2] = v0;
-    } else if (excl + v0 < remaining && remaining <= excl + v0 + v1) {
-      sm.bcast[0] = (unsigned)bin1; sm.bcast[1] = remaining - excl - v0; sm.bcast[2] = v1;
     }
     __syncthreads();
     prefix |= sm.bcast[0] << shift;
