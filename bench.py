@@ -198,7 +198,8 @@ def run_ours(args, wl):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     ctx = cc.Context(local)
-    comp = LayerCompressor(ctx, wl)
+    layout0 = gen.make_layer(wl, layer=100 * rank) if wl.page_size else None
+    comp = LayerCompressor(ctx, wl, layout=layout0)
     work = algorithmic_work(wl)
     peaks = load_peaks()
 
@@ -206,6 +207,8 @@ def run_ours(args, wl):
     dev_sets, host_sets = [], []
     for layer in range(N_LAYER_SETS):
         x = gen.make_layer(wl, layer=layer + 100 * rank)
+        if wl.page_size and layer > 0:
+            gen.repage(x, layout0)          # every layer set uses the page layout of the first
         hs = (to_bf16(x.q_win, "cpu", pin=True), to_bf16(x.k, "cpu", pin=True),
               to_bf16(x.v, "cpu", pin=True), torch.from_numpy(x.prior).pin_memory())
         host_sets.append(hs)
@@ -272,7 +275,11 @@ def run_ours(args, wl):
         elif k == 2:
             cc.cc_topk_select(ctx, d, fused, p_d, comp.idx, comp.count, ws=comp.ws)
         else:
-            cc.cc_compact_kv(ctx, d, k_d, v_d, comp.idx, comp.k_out, comp.v_out)
+            if comp.paged:
+                cc.cc_compact_kv(ctx, d, k_d, v_d, comp.idx, k_d, v_d, comp.free_pages,
+                                 comp.out_page_table)
+            else:
+                cc.cc_compact_kv(ctx, d, k_d, v_d, comp.idx, comp.k_out, comp.v_out)
 
     stage_ms = np.zeros(4)
     stage_reps = max(1, min(args.steps, 200) // N_LAYER_SETS)

@@ -37,29 +37,61 @@ def to_bf16(bits: np.ndarray, device: str = "cuda", pin: bool = False) -> torch.
 
 
 class LayerCompressor:
-    """Pre-allocated state for repeated ``cc_compress_layer`` calls on one geometry
-    (contiguous K/V layout)."""
+    """Pre-allocated state for repeated ``cc_compress_layer`` calls on one geometry.
 
-    def __init__(self, ctx: cc.Context, wl: gen.Workload, mode: int = cc.CC_MODE_BF16):
-        assert wl.page_size == 0, "LayerCompressor handles the contiguous layout"
+    Contiguous K/V: the compacted cache lands in ``k_out`` / ``v_out``.  Paged K/V
+    (``wl.page_size > 0``): ``layout`` supplies the page table, the list of fresh pages and
+    the pool size (a ``LayerInputs`` of the workload); the retained rows are written into
+    fresh pages of the same pool and ``out_page_table`` names them."""
+
+    def __init__(self, ctx: cc.Context, wl: gen.Workload, mode: int = cc.CC_MODE_BF16,
+                 layout: Optional[gen.LayerInputs] = None):
         self.ctx, self.wl = ctx, wl
-        self.desc = desc_from_workload(wl, mode)
         dev = f"cuda:{ctx.device}"
+        self.paged = wl.page_size > 0
         S, hq, hkv, d = len(wl.lens), wl.n_heads_q, wl.n_heads_kv, wl.head_dim
-        n_tot, b_tot = self.desc.n_tot, self.desc.b_tot
         bf = torch.bfloat16
+        if self.paged:
+            if layout is None or layout.page_table is None:
+                raise ValueError("a paged workload needs the page layout (LayerInputs)")
+            ps = wl.page_size
+            self.page_table = torch.from_numpy(layout.page_table).to(dev)
+            self.free_pages = torch.from_numpy(layout.free_pages).to(dev)
+            self.out_pt_stride = max((min(b, n) + ps - 1) // ps
+                                     for b, n in zip(wl.budgets, wl.lens)) + 1
+            self.desc = desc_from_workload(wl, mode, self.page_table, layout.pool_pages,
+                                           self.out_pt_stride)
+            rows = layout.pool_pages * ps
+            self.out_page_table = torch.empty((S, self.out_pt_stride), dtype=torch.int32, device=dev)
+            self.h_out_page_table = torch.empty(self.out_page_table.shape, dtype=torch.int32).pin_memory()
+        else:
+            self.desc = desc_from_workload(wl, mode)
+            rows = self.desc.n_tot
+            self.page_table = self.free_pages = self.out_page_table = None
+        n_tot, b_tot = self.desc.n_tot, self.desc.b_tot
         self.q = torch.empty((S, wl.window, hq, d), dtype=bf, device=dev)
-        self.k = torch.empty((n_tot, hkv, d), dtype=bf, device=dev)
-        self.v = torch.empty((n_tot, hkv, d), dtype=bf, device=dev)
+        self.k = torch.empty((rows, hkv, d), dtype=bf, device=dev)
+        self.v = torch.empty((rows, hkv, d), dtype=bf, device=dev)
         self.prior = torch.empty((n_tot,), dtype=torch.float32, device=dev)
-        self.k_out = torch.empty((b_tot, hkv, d), dtype=bf, device=dev)
-        self.v_out = torch.empty((b_tot, hkv, d), dtype=bf, device=dev)
+        if self.paged:
+            self.k_out = self.v_out = None          # the pool itself receives the retained rows
+        else:
+            self.k_out = torch.empty((b_tot, hkv, d), dtype=bf, device=dev)
+            self.v_out = torch.empty((b_tot, hkv, d), dtype=bf, device=dev)
         self.idx = torch.empty((hkv, b_tot), dtype=torch.int32, device=dev)
         self.count = torch.empty((S, hkv), dtype=torch.int32, device=dev)
         self.ws = ctx.workspace(self.desc)
         # pinned landing buffers for the results
-        self.h_k_out = torch.empty(self.k_out.shape, dtype=bf).pin_memory()
-        self.h_v_out = torch.empty(self.v_out.shape, dtype=bf).pin_memory()
+        if self.paged:
+            ps = wl.page_size
+            n_out_rows = sum((min(b, n) + ps - 1) // ps for b, n in zip(wl.budgets, wl.lens)) * ps
+            self.out_rows = (self.free_pages[: n_out_rows // ps, None].long() * ps
+                             + torch.arange(ps, device=dev)[None, :]).reshape(-1)
+            self.h_k_out = torch.empty((n_out_rows, hkv, d), dtype=bf).pin_memory()
+            self.h_v_out = torch.empty((n_out_rows, hkv, d), dtype=bf).pin_memory()
+        else:
+            self.h_k_out = torch.empty(self.k_out.shape, dtype=bf).pin_memory()
+            self.h_v_out = torch.empty(self.v_out.shape, dtype=bf).pin_memory()
         self.h_idx = torch.empty(self.idx.shape, dtype=torch.int32).pin_memory()
         self.h_count = torch.empty(self.count.shape, dtype=torch.int32).pin_memory()
 
@@ -69,13 +101,20 @@ class LayerCompressor:
 
     @property
     def d2h_bytes(self) -> int:
-        return sum(t.numel() * t.element_size()
-                   for t in (self.k_out, self.v_out, self.idx, self.count))
+        outs = [self.h_k_out, self.h_v_out, self.idx, self.count]
+        if self.paged:
+            outs.append(self.out_page_table)
+        return sum(t.numel() * t.element_size() for t in outs)
 
     def run_device(self, q, k, v, prior) -> None:
-        """Inputs already on the device; outputs land in self.k_out / v_out / idx / count."""
-        cc.cc_compress_layer(self.ctx, self.desc, q, k, v, prior, self.k_out, self.v_out,
-                             self.idx, self.count, ws=self.ws)
+        """Inputs already on the device; outputs land in self.k_out / v_out (contiguous) or in
+        fresh pages of k / v (paged), plus idx / count / out_page_table."""
+        if self.paged:
+            cc.cc_compress_layer(self.ctx, self.desc, q, k, v, prior, k, v, self.idx, self.count,
+                                 self.free_pages, self.out_page_table, ws=self.ws)
+        else:
+            cc.cc_compress_layer(self.ctx, self.desc, q, k, v, prior, self.k_out, self.v_out,
+                                 self.idx, self.count, ws=self.ws)
 
     def run_host(self, q_h, k_h, v_h, prior_h) -> Dict[str, torch.Tensor]:
         """Inputs in (pinned) host memory: copy in, compress, copy the compacted cache back.
@@ -85,9 +124,17 @@ class LayerCompressor:
         self.v.copy_(v_h, non_blocking=True)
         self.prior.copy_(prior_h, non_blocking=True)
         self.run_device(self.q, self.k, self.v, self.prior)
-        self.h_k_out.copy_(self.k_out, non_blocking=True)
-        self.h_v_out.copy_(self.v_out, non_blocking=True)
+        out = {"k_out": self.h_k_out, "v_out": self.h_v_out, "idx": self.h_idx,
+               "count": self.h_count}
+        if self.paged:
+            # the retained rows sit in the fresh pages of the pool: bring just those back
+            self.h_k_out.copy_(self.k[self.out_rows], non_blocking=True)
+            self.h_v_out.copy_(self.v[self.out_rows], non_blocking=True)
+            self.h_out_page_table.copy_(self.out_page_table, non_blocking=True)
+            out["out_page_table"] = self.h_out_page_table
+        else:
+            self.h_k_out.copy_(self.k_out, non_blocking=True)
+            self.h_v_out.copy_(self.v_out, non_blocking=True)
         self.h_idx.copy_(self.idx, non_blocking=True)
         self.h_count.copy_(self.count, non_blocking=True)
-        return {"k_out": self.h_k_out, "v_out": self.h_v_out, "idx": self.h_idx,
-                "count": self.h_count}
+        return out

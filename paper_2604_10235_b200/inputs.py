@@ -219,6 +219,23 @@ def _scatter_into_pages(x: LayerInputs, rng: np.random.Generator) -> None:
     x.pool_pages = pool_pages
 
 
+def repage(x: LayerInputs, ref: LayerInputs) -> None:
+    """Re-scatter the paged K/V of ``x`` so that it uses the page table of ``ref`` (same
+    workload).  Lets several layers share one page layout (in place)."""
+    wl = x.workload
+    ps = wl.page_size
+    k_new, v_new = np.zeros_like(x.k), np.zeros_like(x.v)
+    for s, n_s in enumerate(wl.lens):
+        tok = np.arange(n_s)
+        src = x.page_table[s][tok // ps].astype(np.int64) * ps + tok % ps
+        dst = ref.page_table[s][tok // ps].astype(np.int64) * ps + tok % ps
+        k_new[dst] = x.k[src]
+        if x.v.shape[0]:
+            v_new[dst] = x.v[src]
+    x.k, x.v = k_new, v_new
+    x.page_table, x.free_pages = ref.page_table, ref.free_pages
+
+
 def small_case(seed: int, n: int, window: int, n_heads_q: int, n_heads_kv: int,
                head_dim: int = 128, scale: float = 1.0
                ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
