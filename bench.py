@@ -340,7 +340,7 @@ def run_ours(args, wl):
                              f"{(N_LAYER_SETS - 1) * set_bytes / 1e6:.0f} MB of traffic"},
             "roofline": {"bound": "tensor", "kernel": "score_tc_kernel<1> + score_tc_kernel<2> (the two launches of the score stage)",
                          "achieved": achieved_tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                         "frac": achieved_tf / peaks["bf16_tflops"], "traffic": None,
+                         "frac": achieved_tf / peaks["bf16_tflops"], "traffic": score_traffic(wl),
                          "peak_source": f"{peaks['source']} bf16 burst",
                          "flops_per_launch_pair": work["flops"]},
             "path_roofline": {"t_roof_us": t_roof * 1e6, "t_bytes_us": t_bytes * 1e6,
@@ -359,6 +359,17 @@ def run_ours(args, wl):
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+# DRAM bytes (read + write) of one launch pair of the score stage, from the ncu capture that
+# profiles/score_tc_kernel_llama3_8b.md summarises (llama3_8b: 67.70 + 0.85 MB for pass 1,
+# 68.03 + 0.90 MB for pass 2).  The counters were taken on the kernel as it stands in this tree;
+# other workloads have no capture and report null.
+SCORE_TRAFFIC_BYTES = {"llama3_8b": 137.48e6}
+
+
+def score_traffic(wl):
+    return SCORE_TRAFFIC_BYTES.get(wl.name)
 
 
 def main():
