@@ -44,10 +44,15 @@ namespace cc {
 
 namespace {
 
-constexpr int kThreads = 608;                             // TMA, 2 MMA issuers, 16 epilogue warps
-constexpr int kMmaWarpB = 18;                             // second MMA issuer
-constexpr int kIssuers = 2;
+#ifndef CC_ISSUERS
+#define CC_ISSUERS 2
+#endif
+constexpr int kIssuers = CC_ISSUERS;                      // 1 or 2
 constexpr int kEpiWarps = 16;
+constexpr int kThreads = (1 + kIssuers + kEpiWarps) * 32; // TMA, the MMA issuers, 16 epilogue warps
+constexpr int kMmaWarpB = 2 + kEpiWarps;                  // second MMA issuer (the last warp), if any
+static_assert(kIssuers == 1 || kIssuers == 2, "every warp of the CTA needs a role");
+static_assert(kThreads / 32 == kMmaWarpB + kIssuers - 1, "warps 0, 1, the epilogue warps, the second issuer");
 constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kMaxStages = 6;
 constexpr uint32_t kPanelBytes = kTileKeys * 128;        // one 64-channel half of a K tile
@@ -391,7 +396,8 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
       mbar_init(smem_u32(&misc->bar.acc_empty[i]), 4);       // the four warps of a set
     }
     for (int i = 0; i < 8; ++i)
-      for (int j = 0; j < 4; ++j) mbar_init(smem_u32(&misc->bar.u_full[i][j]), kSets - 1);
+      for (int j = 0; j < 4; ++j)        // one arrival per set that hands its partial sums over
+        mbar_init(smem_u32(&misc->bar.u_full[i][j]), P.n_sub > 1 ? P.n_sub - 1 : 1);
     misc->abort_flag = 0;
     fence_barrier_init();
   }
@@ -467,7 +473,7 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
         if (++stage == P.n_stages) { stage = 0; phase ^= 1; }
       }
     }
-  } else if (warp == 1 || warp == kMmaWarpB) {
+  } else if (warp == 1 || (kIssuers == 2 && warp == kMmaWarpB)) {
     // ================================================================ MMA issuers
     // The serial instruction stream of a thread that issues tcgen05.mma (waits, descriptor
     // words, eight multiplications and a commit per item) is long, so there are two issuers;
@@ -512,7 +518,7 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
         const uint32_t k_lo = k_lo0 + (uint32_t)stage * (kStageBytes >> 4);
 #pragma unroll 1
         for (int sub = 0; sub < P.n_sub; ++sub, ++item) {
-          if ((int)((item >> 1) & 1u) != my_half) continue;
+          if (kIssuers == 2 && (int)((item >> 1) & 1u) != my_half) continue;
           const uint32_t buf = item & (kBufs - 1);
           const uint32_t par = ((item >> 2) & 1u) ^ 1u;
           if (!mbar_try_wait(acce0 + 8u * buf, par) &&
@@ -559,7 +565,7 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
         }
       }
     }
-  } else {
+  } else if (warp >= 2 && warp < 2 + kEpiWarps) {
     // ================================================================ epilogue warps
     const int ew = warp - 2;                 // 0..15
     const int quad = warp & 3;               // TMEM lane quadrant this warp may read
@@ -572,7 +578,6 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
     TileCursor cur;
     cur.locate(bt, g.hkv, t_begin);
     int cur_problem = -1;
-    uint32_t item = 0;
     bool dead = false;      // after a failed wait: keep the loop structure (and its barriers), skip the work
     float run_m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
     float run_l[4] = {0.f, 0.f, 0.f, 0.f};
@@ -582,10 +587,15 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
 #pragma unroll
       for (int rb = 0; rb < 4; ++rb) {
         if (rb >= P.n_sub) break;
-        misc->xchg[set][rb * 128 + row_in_tile] = make_float2(run_m[rb], run_l[rb]);
-        run_m[rb] = -INFINITY;
-        run_l[rb] = 0.f;
+        // a set whose row block never changes keeps its state in slot 0
+        const int own = P.n_sub == 3 ? rb : (rb == set % P.n_sub ? 0 : -1);
+        float2 st = make_float2(-INFINITY, 0.f);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) if (k == own) st = make_float2(run_m[k], run_l[k]);
+        misc->xchg[set][rb * 128 + row_in_tile] = st;
       }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) { run_m[k] = -INFINITY; run_l[k] = 0.f; }
       epi_barrier();
       for (int row = etid; row < P.rows_pad; row += kEpiThreads) {
         float m = -INFINITY;
@@ -602,107 +612,118 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
       epi_barrier();
     };
 
-    // the cursor is walked only where the (sequence, head) changes; in between a countdown and
-    // a running key offset describe the tile
-    int left = 0, key0 = 0, n_cur = 0;
-    int64_t out_base = 0;
-    for (int t = t_begin; t < t_end; ++t, key0 += kTileKeys, --left) {
-      if (left == 0) {
-        if (cur_problem >= 0) {
-          cur.local = cur.n_tiles - 1;
-          cur.advance(bt, g.hkv);
-        }
-        const SeqInfo& sq = bt.seq[cur.s];
-        if (PASS == 1) {
-          if (cur_problem >= 0) flush_partial(cur_problem);
-        } else {
-          // merge the spans' (max, sum) of the new (sequence, head) into -L_r: the spans are
-          // dealt round-robin to the threads that share a row, all loads of a thread are issued
-          // before the first use, and the threads of a row meet through shared memory
-          epi_barrier();
-          const int first_tile = g.hkv * sq.tile_off + cur.h * sq.n_tiles;
-          const int b0 = cta_of_tile(first_tile, P), b1 = cta_of_tile(first_tile + sq.n_tiles - 1, P);
-          const int problem = cur.problem(g.hkv);
-          const int ways = max(1, min(4, kEpiThreads / P.rows_pad));    // threads per row
-          const int per_sweep = kEpiThreads / ways;                     // rows per sweep
-          float2* fold = &misc->xchg[0][0];          // no tile is in flight here, the union is free
-          for (int base = 0; base < P.rows_pad; base += per_sweep) {
-            const int row = base + etid % per_sweep, way = etid / per_sweep;
-            float m = -INFINITY, l = 0.f;
-            if (row < P.rows_pad) {
-              for (int b = b0 + way; b <= b1; b += 8 * ways) {
-                float2 pr[8];
+    // pass 2 (first_tile = the (sequence, head)'s first tile, tb = its first tile in this span):
+    auto merge_lse = [&](const SeqInfo& sq, int first_tile, int tb) {
+      // merge the spans' (max, sum) of the new (sequence, head) into -L_r: the spans are
+      // dealt round-robin to the threads that share a row, all loads of a thread are issued
+      // before the first use, and the threads of a row meet through shared memory
+      epi_barrier();
+      const int b0 = cta_of_tile(first_tile, P), b1 = cta_of_tile(first_tile + sq.n_tiles - 1, P);
+      const int problem = cur.problem(g.hkv);
+      const int ways = max(1, min(4, kEpiThreads / P.rows_pad));    // threads per row
+      const int per_sweep = kEpiThreads / ways;                     // rows per sweep
+      float2* fold = &misc->xchg[0][0];          // no tile is in flight here, the union is free
+      for (int base = 0; base < P.rows_pad; base += per_sweep) {
+        const int row = base + etid % per_sweep, way = etid / per_sweep;
+        float m = -INFINITY, l = 0.f;
+        if (row < P.rows_pad) {
+          for (int b = b0 + way; b <= b1; b += 8 * ways) {
+            float2 pr[8];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                  const int bb = b + k * ways;
-                  pr[k] = bb <= b1 ? P.part[(int64_t)(bb + problem) * P.rows_pad + row]
-                                   : make_float2(-INFINITY, 0.f);
-                }
+            for (int k = 0; k < 8; ++k) {
+              const int bb = b + k * ways;
+              pr[k] = bb <= b1 ? P.part[(int64_t)(bb + problem) * P.rows_pad + row]
+                               : make_float2(-INFINITY, 0.f);
+            }
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                  if (pr[k].y > 0.f) {
-                    const float mn = fmaxf(m, pr[k].x);
-                    l = l * ex2(m - mn) + pr[k].y * ex2(pr[k].x - mn);
-                    m = mn;
-                  }
-                }
+            for (int k = 0; k < 8; ++k) {
+              if (pr[k].y > 0.f) {
+                const float mn = fmaxf(m, pr[k].x);
+                l = l * ex2(m - mn) + pr[k].y * ex2(pr[k].x - mn);
+                m = mn;
               }
-              if (ways > 1) fold[etid] = make_float2(m, l);
             }
-            if (ways > 1) epi_barrier();
-            if (row < P.rows_pad && way == 0) {
-              for (int k = 1; k < ways; ++k) {
-                const float2 o = fold[k * per_sweep + etid];
-                if (o.y > 0.f) {
-                  const float mn = fmaxf(m, o.x);
-                  l = l * ex2(m - mn) + o.y * ex2(o.x - mn);
-                  m = mn;
-                }
-              }
-              const float lc = m + log2f(l);
-              const int gq = row % g.group, tq = row / g.group;     // row = t * G + g
-              const bool real = tq < g.window;
-              misc->neg_lc[row] = real ? -lc : -1.0e4f;
-              if (real && P.lse != nullptr && t == first_tile)
-                P.lse[((int64_t)cur.s * g.hq + cur.h * g.group + gq) * g.window + tq] = lc * kLn2;
-            }
-            if (ways > 1) epi_barrier();
           }
-          epi_barrier();
+          if (ways > 1) fold[etid] = make_float2(m, l);
         }
-        cur_problem = cur.problem(g.hkv);
-        left = cur.n_tiles - cur.local;
-        key0 = cur.local * kTileKeys;
-        n_cur = sq.n;
-        out_base = (int64_t)cur.h * bt.n_tot + sq.tok_off;
+        if (ways > 1) epi_barrier();
+        if (row < P.rows_pad && way == 0) {
+          for (int k = 1; k < ways; ++k) {
+            const float2 o = fold[k * per_sweep + etid];
+            if (o.y > 0.f) {
+              const float mn = fmaxf(m, o.x);
+              l = l * ex2(m - mn) + o.y * ex2(o.x - mn);
+              m = mn;
+            }
+          }
+          const float lc = m + log2f(l);
+          const int gq = row % g.group, tq = row / g.group;     // row = t * G + g
+          const bool real = tq < g.window;
+          misc->neg_lc[row] = real ? -lc : -1.0e4f;
+          if (real && P.lse != nullptr && tb == first_tile)
+            P.lse[((int64_t)cur.s * g.hq + cur.h * g.group + gq) * g.window + tq] = lc * kLn2;
+        }
+        if (ways > 1) epi_barrier();
       }
-      const uint32_t item0 = item;          // first item of the tile
-      if (((uint32_t)(set - (int)(item0 & (kBufs - 1))) & (kBufs - 1)) >= (uint32_t)P.n_sub) {
-        item += (uint32_t)P.n_sub;          // none of the tile's items is this set's
-        continue;
-      }
-      const int valid = min(kTileKeys, n_cur - key0);
-      float u_acc = 0.f;
+      epi_barrier();
+    };
 
-#pragma unroll 1
-      for (int sub = 0; sub < P.n_sub; ++sub, ++item) {
-        const uint32_t buf = item & (kBufs - 1);
-        if ((int)buf != set) continue;
-        if (!dead) {
-          // one lane probes; the vote doubles as the hand-over to the other lanes
-          const bool got = lane != 0 || wait_bar(pipe, &misc->bar.acc_full[buf], (item >> 2) & 1u, 30);
+    // A set works on every fourth item of the span, item = (tile - t_begin) * n_sub + sub, and
+    // steps from one of its items to the next by a precomputed (tiles, subs) stride; the
+    // cursor is walked only where the (sequence, head) changes.  Buffer = set, and the phase
+    // of its barrier flips with every item.
+    const int n_sub = P.n_sub;
+    const int dt = kSets / n_sub, ds = kSets % n_sub;
+    const bool rotating = ds != 0;          // the set's row block changes from item to item
+    int sub = set % n_sub, t = t_begin + set / n_sub;
+    uint32_t par = 0;
+    int prob_end = t_begin, first_tile = 0, n_cur = 0;
+    int64_t out_base = 0;
+    const uint32_t full_bar = smem_u32(&misc->bar.acc_full[set]);
+    const uint32_t empty_bar = smem_u32(&misc->bar.acc_empty[set]);
+    const uint32_t acc_addr = lane_addr + (uint32_t)set * kBufCols;
+    for (;;) {
+      if (t >= prob_end) {
+        bool done = false;
+        do {
+          if (PASS == 1 && cur_problem >= 0) flush_partial(cur_problem);
+          if (prob_end >= t_end) { done = true; break; }
+          if (cur_problem >= 0) {
+            cur.local = cur.n_tiles - 1;
+            cur.advance(bt, g.hkv);
+          }
+          const SeqInfo& sq = bt.seq[cur.s];
+          first_tile = g.hkv * sq.tile_off + cur.h * sq.n_tiles;
+          if (PASS == 2) merge_lse(sq, first_tile, prob_end);
+          cur_problem = cur.problem(g.hkv);
+          prob_end = min(t_end, first_tile + sq.n_tiles);
+          n_cur = sq.n;
+          out_base = (int64_t)cur.h * bt.n_tot + sq.tok_off;
+        } while (t >= prob_end);
+        if (done) break;
+      }
+      const int key0 = (t - first_tile) * kTileKeys;
+      const int valid = min(kTileKeys, n_cur - key0);
+      if (!dead) {
+        // every lane probes once; only when the buffer is not full yet does one lane wait
+        if (!__all_sync(0xffffffffu, mbar_try_wait(full_bar, par))) {
+          const bool got = lane != 0 || wait_bar(pipe, &misc->bar.acc_full[set], par, 30);
           dead = !__all_sync(0xffffffffu, got);
         }
-        if (dead) continue;
+      }
+      par ^= 1u;
+      float u_acc = 0.f;
+      if (!dead) {
         tc_fence_after();
-        const uint32_t acc_addr = lane_addr + buf * kBufCols;
         uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
         uint32_t v[32];
         if (PASS == 1) {
           // thread = query row (sub * 128 + row_in_tile); columns = the 128 keys of the tile
-          float m_run = -INFINITY, l_run = 0.f;
+          float m_run = run_m[0], l_run = run_l[0];
+          if (rotating) {
 #pragma unroll
-          for (int rb = 0; rb < 4; ++rb) if (rb == sub) { m_run = run_m[rb]; l_run = run_l[rb]; }
+            for (int rb = 1; rb < 4; ++rb) if (rb == sub) { m_run = run_m[rb]; l_run = run_l[rb]; }
+          }
 #pragma unroll 1
           for (int cc0 = 0; cc0 < kTileKeys; cc0 += 32) {
             tmem_ld32(acc_addr + (uint32_t)cc0, v);
@@ -710,7 +731,7 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
             if (cc0 + 32 == kTileKeys) {             // last read of the buffer: hand it back
               tc_fence_before();
               __syncwarp();
-              if (lane == 0) mbar_arrive(smem_u32(&misc->bar.acc_empty[buf]));
+              if (lane == 0) mbar_arrive(empty_bar);
             }
             if (cc0 >= valid) continue;
             if (cc0 + 32 > valid) {
@@ -729,8 +750,13 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
             exp_accumulate<false, 32>(v, c2, pack2(-m_run, -m_run), nullptr, acc);
           }
           l_run += acc_total(acc);
+          if (rotating) {
 #pragma unroll
-          for (int rb = 0; rb < 4; ++rb) if (rb == sub) { run_m[rb] = m_run; run_l[rb] = l_run; }
+            for (int rb = 0; rb < 4; ++rb) if (rb == sub) { run_m[rb] = m_run; run_l[rb] = l_run; }
+          } else {
+            run_m[0] = m_run;
+            run_l[0] = l_run;
+          }
         } else {
           // thread = key (key0 + row_in_tile); columns = the query rows of this chunk
           const int c0 = sub * P.sub_cols;
@@ -743,49 +769,46 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
             if (cc0 + 32 >= nc) {
               tc_fence_before();
               __syncwarp();
-              if (lane == 0) mbar_arrive(smem_u32(&misc->bar.acc_empty[buf]));
+              if (lane == 0) mbar_arrive(empty_bar);
             }
             if (cc0 + 32 <= nc) exp_accumulate<true, 32>(v, c2, 0ull, nl + cc0, acc);
             else                exp_accumulate<true, 16>(v, c2, 0ull, nl + cc0, acc);
           }
-          u_acc += acc_total(acc);
+          u_acc = acc_total(acc);
         }
       }
-      if (PASS == 2 && P.n_sub > 1) {
-        // The sets that hold partial sums of the tile (one per item) meet through shared
-        // memory: the set that drained the tile's last item adds the others' sums and stores.
-        // kSets - 1 arrivals complete a (slot, quadrant); the storing warp tops up what is
-        // missing when the tile has fewer than four items.  Eight slots: a slot is written again
-        // only after the accumulator hand-shake has forced the reader past the tile it belongs to.
-        const int n_items = (int)(item - item0);                  // 2..4
-        const int last_set = (int)((item - 1u) & (kBufs - 1));
-        const bool worked = ((uint32_t)(set - (int)(item0 & (kBufs - 1))) & (kBufs - 1)) < (uint32_t)n_items;
-        const int slot = t & 7;
-        if (worked && set != last_set) {
-          misc->u_part[slot][set][row_in_tile] = u_acc;
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&misc->bar.u_full[slot][quad]));
-        } else if (set == last_set) {
-          if (lane == 0 && n_items < kSets)
-            mbar_arrive_n(smem_u32(&misc->bar.u_full[slot][quad]), (uint32_t)(kSets - n_items));
-          if (!dead) {
-            const bool got = lane != 0 || wait_bar(pipe, &misc->bar.u_full[slot][quad],
-                                                   (uint32_t)((t - t_begin) >> 3) & 1u, 31);
-            dead = !__all_sync(0xffffffffu, got);
+      if (PASS == 2) {
+        if (n_sub > 1) {
+          // The sets that hold partial sums of the tile (one per item) meet through shared
+          // memory: the set that drained the tile's last item adds the others' sums and stores;
+          // n_sub - 1 arrivals complete a (slot, quadrant).  Eight slots: a slot is written
+          // again only after the accumulator hand-shake has forced the reader past the tile it
+          // belongs to.
+          const int slot = t & 7;
+          if (sub != n_sub - 1) {
+            misc->u_part[slot][sub][row_in_tile] = u_acc;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&misc->bar.u_full[slot][quad]));
+          } else {
+            if (!dead) {
+              const bool got = lane != 0 || wait_bar(pipe, &misc->bar.u_full[slot][quad],
+                                                     (uint32_t)((t - t_begin) >> 3) & 1u, 31);
+              dead = !__all_sync(0xffffffffu, got);
+            }
+            if (!dead && row_in_tile < valid) {
+              float u = u_acc;
+              for (int k = 0; k < n_sub - 1; ++k) u += misc->u_part[slot][k][row_in_tile];
+              P.scores[out_base + key0 + row_in_tile] = u;
+            }
           }
-          if (!dead && row_in_tile < valid) {
-            float u = u_acc;
-            for (int k = 1; k < n_items; ++k)
-              u += misc->u_part[slot][(last_set + kSets - k) & (kSets - 1)][row_in_tile];
-            P.scores[out_base + key0 + row_in_tile] = u;
-          }
-        }
-      } else if (PASS == 2) {
-        if ((int)(item0 & (kBufs - 1)) == set && !dead && row_in_tile < valid)
+        } else if (!dead && row_in_tile < valid) {
           P.scores[out_base + key0 + row_in_tile] = u_acc;
+        }
       }
+      sub += ds;
+      t += dt;
+      if (sub >= n_sub) { sub -= n_sub; ++t; }
     }
-    if (PASS == 1 && cur_problem >= 0) flush_partial(cur_problem);
   }
 
   // ---------------------------------------------------------------- teardown
