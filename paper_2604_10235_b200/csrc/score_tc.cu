@@ -414,60 +414,64 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
 
   if (warp == 0) {
     // ================================================================ TMA producer
-    if (lane == 0) {
+    // The whole warp walks the tile list; lane 0 waits and issues the copies of contiguous K.
+    // With a paged cache every lane owns one page of the tile: it reads the page id (before the
+    // wait for the stage, so the load is covered), checks it and issues the two copies of its
+    // page, so the page-table look-ups of a tile are one parallel load instead of a chain.
+    {
       TileCursor cur;
       cur.locate(bt, g.hkv, t_begin);
       int stage = 0, cur_problem = -1;
       uint32_t phase = 0, qe_phase = 0;
+      const int ps = bt.page_size;
       for (int t = t_begin; t < t_end; ++t, cur.advance(bt, g.hkv)) {
         const SeqInfo& sq = bt.seq[cur.s];
         if (cur.problem(g.hkv) != cur_problem) {
           if (cur_problem >= 0) {
-            if (!wait_bar(pipe, &misc->bar.q_empty, qe_phase, 10)) break;
+            const bool got = lane != 0 || wait_bar(pipe, &misc->bar.q_empty, qe_phase, 10);
+            if (!__all_sync(0xffffffffu, got)) break;
             qe_phase ^= 1;
           }
           cur_problem = cur.problem(g.hkv);
-          const uint32_t qb = smem_u32(&misc->bar.q_full);
-          mbar_expect_tx(qb, q_bytes);
-          tma_load_4d(smem_u32(q_smem), &q_map, qb, 0, cur.h * g.group, 0, cur.s);
-          tma_load_4d(smem_u32(q_smem) + q_panel, &q_map, qb, 64, cur.h * g.group, 0, cur.s);
+          if (lane == 0) {
+            const uint32_t qb = smem_u32(&misc->bar.q_full);
+            mbar_expect_tx(qb, q_bytes);
+            tma_load_4d(smem_u32(q_smem), &q_map, qb, 0, cur.h * g.group, 0, cur.s);
+            tma_load_4d(smem_u32(q_smem) + q_panel, &q_map, qb, 64, cur.h * g.group, 0, cur.s);
+          }
         }
-        if (!wait_bar(pipe, &misc->bar.empty[stage], phase ^ 1, 11)) break;
+        const int key0 = cur.local * kTileKeys;
+        int page_id = -1;
+        bool mine = false;               // this lane owns a page of the tile
+        if (ps > 0) {
+          const int valid = min(kTileKeys, sq.n - key0);
+          mine = lane < (valid + ps - 1) / ps;
+          if (mine) page_id = g.page_table[(int64_t)cur.s * g.page_table_stride + key0 / ps + lane];
+        }
+        {
+          const bool got = lane != 0 || wait_bar(pipe, &misc->bar.empty[stage], phase ^ 1, 11);
+          if (!__all_sync(0xffffffffu, got)) break;
+        }
         const uint32_t fb = smem_u32(&misc->bar.full[stage]);
         const uint32_t dst = smem_u32(k_smem) + (uint32_t)stage * kStageBytes;
-        const int key0 = cur.local * kTileKeys;
-        if (bt.page_size == 0) {
-          mbar_expect_tx(fb, kStageBytes);
-          tma_load_3d(dst, &k_map, fb, 0, cur.h, sq.tok_off + key0);
-          tma_load_3d(dst + kPanelBytes, &k_map, fb, 64, cur.h, sq.tok_off + key0);
-        } else {
-          const int ps = bt.page_size;
-          const int valid = min(kTileKeys, sq.n - key0);
-          const int n_pages = (valid + ps - 1) / ps;
-          const int32_t* pt = g.page_table + (int64_t)cur.s * g.page_table_stride + key0 / ps;
-          int ids[16];
-          int good = 0;
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            ids[i] = -1;
-            if (i < n_pages) {
-              ids[i] = pt[i];
-              if (ids[i] < 0 || ((int64_t)ids[i] + 1) * ps > P.pool_rows) {
-                ids[i] = -1;
-                report_error(status, CC_ERR_DEVICE_FLAG, 12);
-              } else {
-                ++good;
-              }
-            }
+        if (ps == 0) {
+          if (lane == 0) {
+            mbar_expect_tx(fb, kStageBytes);
+            tma_load_3d(dst, &k_map, fb, 0, cur.h, sq.tok_off + key0);
+            tma_load_3d(dst + kPanelBytes, &k_map, fb, 64, cur.h, sq.tok_off + key0);
           }
-          mbar_expect_tx(fb, (uint32_t)good * (uint32_t)ps * 256u);
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            if (ids[i] >= 0) {
-              const uint32_t off = (uint32_t)i * (uint32_t)ps * 128u;
-              tma_load_3d(dst + off, &k_map, fb, 0, cur.h, ids[i] * ps);
-              tma_load_3d(dst + kPanelBytes + off, &k_map, fb, 64, cur.h, ids[i] * ps);
-            }
+        } else {
+          const bool good = mine && page_id >= 0 && ((int64_t)page_id + 1) * ps <= P.pool_rows;
+          if (mine && !good) report_error(status, CC_ERR_DEVICE_FLAG, 12);
+          const unsigned good_mask = __ballot_sync(0xffffffffu, good);
+          // the stage completes when the bytes of the good pages have landed; the expectation is
+          // registered before any lane issues a copy
+          if (lane == 0) mbar_expect_tx(fb, (uint32_t)__popc(good_mask) * (uint32_t)ps * 256u);
+          __syncwarp();
+          if (good) {
+            const uint32_t off = (uint32_t)lane * (uint32_t)ps * 128u;
+            tma_load_3d(dst + off, &k_map, fb, 0, cur.h, page_id * ps);
+            tma_load_3d(dst + kPanelBytes + off, &k_map, fb, 64, cur.h, page_id * ps);
           }
         }
         if (++stage == P.n_stages) { stage = 0; phase ^= 1; }
