@@ -187,6 +187,7 @@ def run_ours(args, wl):
     import torch.distributed as dist
     from paper_2604_10235_b200 import binding as cc
     from paper_2604_10235_b200 import inputs as gen
+    from paper_2604_10235_b200 import sharding
     from paper_2604_10235_b200.api import LayerCompressor, to_bf16
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -198,16 +199,17 @@ def run_ours(args, wl):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     ctx = cc.Context(local)
-    layout0 = gen.make_layer(wl, layer=100 * rank) if wl.page_size else None
+    layers = sharding.rank_layers(rank, N_LAYER_SETS)
+    layout0 = gen.make_layer(wl, layer=layers[0]) if wl.page_size else None
     comp = LayerCompressor(ctx, wl, layout=layout0)
     work = algorithmic_work(wl)
     peaks = load_peaks()
 
     # inputs: N_LAYER_SETS layers, resident in HBM before timing, plus pinned host copies
     dev_sets, host_sets = [], []
-    for layer in range(N_LAYER_SETS):
-        x = gen.make_layer(wl, layer=layer + 100 * rank)
-        if wl.page_size and layer > 0:
+    for i, layer in enumerate(layers):
+        x = gen.make_layer(wl, layer=layer)
+        if wl.page_size and i > 0:
             gen.repage(x, layout0)          # every layer set uses the page layout of the first
         hs = (to_bf16(x.q_win, "cpu", pin=True), to_bf16(x.k, "cpu", pin=True),
               to_bf16(x.v, "cpu", pin=True), torch.from_numpy(x.prior).pin_memory())
@@ -216,16 +218,11 @@ def run_ours(args, wl):
     set_bytes = sum(t.numel() * t.element_size() for t in dev_sets[0])
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        sharding.barrier(world)
         torch.cuda.synchronize()
 
     def max_over_ranks(ms: float) -> float:
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return sharding.max_over_ranks(ms, world, "cuda")
 
     # ---- device-resident timing: the fused call on each of the layer sets is captured once in
     # a CUDA graph (one replay = N_LAYER_SETS steps), so the timed region holds kernel time and
@@ -260,7 +257,7 @@ def run_ours(args, wl):
     if status != 0:
         raise RuntimeError(f"device status {status} after the timed region")
     ms_step = ms_total / args.steps
-    value = world * work["tokens"] / (ms_step * 1e-3)
+    value = sharding.job_throughput(work["tokens"], world, ms_step)
 
     # ---- per-stage durations: each stage entry point captured the same way and replayed
     d = comp.desc
@@ -319,7 +316,7 @@ def run_ours(args, wl):
     e1.record()
     barrier()
     ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / n_e2e
-    e2e_value = world * work["tokens"] / (ms_e2e * 1e-3)
+    e2e_value = sharding.job_throughput(work["tokens"], world, ms_e2e)
 
     if rank == 0:
         cpu = None

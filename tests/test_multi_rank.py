@@ -1,0 +1,58 @@
+"""The multi-process plumbing on CPU: two gloo ranks take disjoint layer streams, meet at the
+barrier, and agree on the slowest rank's time and on the job throughput.  No GPU needed."""
+import os
+import socket
+
+import numpy as np
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from paper_2604_10235_b200 import inputs as gen
+from paper_2604_10235_b200 import sharding
+
+
+def _free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _rank_main(rank: int, world: int, port: int, out) -> None:
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        layers = sharding.rank_layers(rank, 4)
+        wl = gen.workloads()["tiny"]
+        x = gen.make_layer(wl, layer=layers[0], with_v=False)
+        sharding.barrier(world)
+        ms_local = 2.0 + rank                                  # rank 1 is the slow one
+        ms = sharding.max_over_ranks(ms_local, world)
+        out.put((rank, layers, int(x.k.astype(np.int64).sum()), ms,
+                 sharding.job_throughput(1000, world, ms)))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_shard_layers_and_reduce_timings():
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_rank_main, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = sorted(out.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    (_, l0, sum0, ms0, v0), (_, l1, sum1, ms1, v1) = got
+    assert not set(l0) & set(l1)                  # disjoint layer streams
+    assert sum0 != sum1                           # and therefore different synthetic inputs
+    assert ms0 == ms1 == 3.0                      # everyone reports the slowest rank's time
+    assert v0 == v1 == 2 * 1000 / 3.0e-3          # whole-job tokens/s: both ranks' tokens
+
+
+def test_single_rank_needs_no_process_group():
+    assert sharding.max_over_ranks(1.5, 1) == 1.5
+    sharding.barrier(1)
+    assert sharding.rank_layers(3, 2) == [300, 301]
+    assert abs(sharding.job_throughput(32768, 1, 0.0689) - 32768 / 0.0689e-3) < 1e-3
