@@ -25,12 +25,18 @@ What each function follows:
                         (remaining capacity filled by top-ranked attention scores).
 * ``compact_kv``      - the retained K/V rows in original order (Section 4.6: chunks
                         keep their original position indices).
+* ``structural_score`` - Section 5.3, caption of the bug-localization table: the fraction
+                        of structurally critical tokens that a retained set contains
+                        (the table averages it over layers and chunks; the average is
+                        the caller's).
 
 Readings of the paper that are choices rather than statements of it ("parity
 unpinned" by the paper, pinned here only by self-consistency tests):
   - the normalisation of the attention term inside ``fuse_prior`` (alpha is a free
     caller-chosen factor);
-  - the edge rule of average pooling (zero padding, always divide by the width).
+  - the edge rule of average pooling (zero padding, always divide by the width);
+  - ``structural_score`` of a sequence without structurally critical tokens is taken
+    as 1 (nothing could be lost); the paper does not say.
 """
 from __future__ import annotations
 
@@ -215,6 +221,18 @@ def compact_kv(k_bits: np.ndarray, v_bits: np.ndarray, idx: Sequence[np.ndarray]
     k_out = [k_bits[np.asarray(ix, dtype=np.int64), h, :] for h, ix in enumerate(idx)]
     v_out = [v_bits[np.asarray(ix, dtype=np.int64), h, :] for h, ix in enumerate(idx)]
     return k_out, v_out
+
+
+# --------------------------------------------------------------------------- Str. Score
+def structural_score(idx: np.ndarray, prior: np.ndarray, threshold: float
+                     ) -> Tuple[float, int, int]:
+    """Fraction of the structurally critical tokens {j : prior[j] >= threshold} that the
+    retained index set ``idx`` (entries < 0 are padding) contains; also the two counts
+    (retained critical tokens, critical tokens).  Defined as 1.0 when there are none."""
+    critical = set(int(j) for j in np.flatnonzero(np.asarray(prior, dtype=np.float64) >= threshold))
+    kept = set(int(j) for j in np.asarray(idx).ravel() if j >= 0)
+    hit = len(critical & kept)
+    return (hit / len(critical) if critical else 1.0), hit, len(critical)
 
 
 # --------------------------------------------------------------------------- paged layout

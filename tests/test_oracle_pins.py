@@ -327,3 +327,49 @@ def test_workload_recipe_statistics():
     rows = orc.paged_rows(x.page_table[1], 70, 16)
     np.testing.assert_array_equal(x.k[rows], y.k[40:110])                  # same bits, scattered
     assert len(set(x.free_pages.tolist()) & set(x.page_table[x.page_table >= 0].tolist())) == 0
+
+
+# --------------------------------------------------------------------------- Str. Score
+def test_structural_score_hand_values():
+    """Section 5.3 (table caption): fraction of structurally critical tokens retained.
+    Worked by hand: critical = {0, 2, 3, 6}; a retained set {0, 1, 3} holds two of the four."""
+    prior = np.array([1, 0, 1, 1, 0, 0, 1], dtype=np.float32)
+    frac, hit, tot = orc.structural_score(np.array([0, 1, 3, -1]), prior, 0.5)
+    assert (frac, hit, tot) == (0.5, 2, 4)
+    assert orc.structural_score(np.array([0, 2, 3, 6]), prior, 0.5) == (1.0, 4, 4)
+    assert orc.structural_score(np.array([1, 4, 5]), prior, 0.5) == (0.0, 0, 4)
+    # no critical token at all: nothing can be lost
+    assert orc.structural_score(np.array([1, 4]), prior, 2.0) == (1.0, 0, 0)
+    # the threshold is inclusive, like the protection rule of the selection
+    assert orc.structural_score(np.array([0]), np.array([0.5, 0.49]), 0.5) == (1.0, 1, 1)
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_structural_score_vs_counting_loop(seed):
+    rng = np.random.Generator(np.random.PCG64(900 + seed))
+    n = 300
+    prior = (rng.random(n) < 0.2).astype(np.float32)
+    idx = np.sort(rng.choice(n, size=60, replace=False))
+    hit = tot = 0
+    for j in range(n):
+        if prior[j] >= 0.5:
+            tot += 1
+            hit += int(j in idx)
+    assert orc.structural_score(idx, prior, 0.5) == (hit / tot, hit, tot)
+
+
+def test_structural_score_is_one_when_protected_tokens_fit_the_budget():
+    """Section 4.4 "Token-level protection": protected tokens are kept first, so when they fit
+    the budget the retained set of every head contains all of them."""
+    wl = gen.workloads()["tiny"]
+    x = gen.make_layer(wl)
+    res = orc.compress_sequence(x.q_win[0], x.k, None, x.prior, wl.n_heads_kv, wl.pool_kind,
+                                wl.pool_size, wl.budget, wl.alpha, wl.beta, wl.force_threshold)
+    assert int((x.prior >= wl.force_threshold).sum()) <= wl.budget
+    for h in range(wl.n_heads_kv):
+        frac, hit, tot = orc.structural_score(res["idx"][h], x.prior, wl.force_threshold)
+        assert frac == 1.0 and hit == tot > 0
+    # without protection (threshold out of reach for the selection) attention alone keeps fewer
+    res2 = orc.compress_sequence(x.q_win[0], x.k, None, x.prior, wl.n_heads_kv, wl.pool_kind,
+                                 wl.pool_size, wl.budget, wl.alpha, wl.beta, float("inf"))
+    assert orc.structural_score(res2["idx"][0], x.prior, wl.force_threshold)[0] < 1.0
