@@ -271,16 +271,20 @@ def run_ours(args, wl):
             cc.cc_fuse_prior_pool(ctx, d, scores, p_d, fused)
         elif k == 2:
             cc.cc_topk_select(ctx, d, fused, p_d, comp.idx, comp.count, ws=comp.ws)
-        else:
+        elif k == 3:
             if comp.paged:
                 cc.cc_compact_kv(ctx, d, k_d, v_d, comp.idx, k_d, v_d, comp.free_pages,
                                  comp.out_page_table)
             else:
                 cc.cc_compact_kv(ctx, d, k_d, v_d, comp.idx, comp.k_out, comp.v_out)
+        else:
+            # not part of a step: the retained fraction of the structurally critical tokens
+            cc.cc_structural_score(ctx, d, comp.idx, p_d, wl.force_threshold, str_score)
 
-    stage_ms = np.zeros(4)
+    str_score = torch.empty((len(wl.lens), wl.n_heads_kv), device="cuda")
+    stage_ms = np.zeros(5)
     stage_reps = max(1, min(args.steps, 200) // N_LAYER_SETS)
-    for k in range(4):
+    for k in range(5):
         for j in range(N_LAYER_SETS):
             stage_call(k, *dev_sets[j])
         torch.cuda.synchronize()
@@ -345,7 +349,9 @@ def run_ours(args, wl):
                               "frac": t_roof / (ms_step * 1e-3), "bytes": work["bytes"],
                               "flops": work["flops"], "hbm_peak_gbs": peaks["hbm_gbs"]},
             "stage_us": {"score": stage_ms[0] * 1e3, "fuse_pool": stage_ms[1] * 1e3,
-                         "select": stage_ms[2] * 1e3, "compact": stage_ms[3] * 1e3},
+                         "select": stage_ms[2] * 1e3, "compact": stage_ms[3] * 1e3,
+                         "str_score_diagnostic": stage_ms[4] * 1e3},
+            "str_score": [round(float(v), 4) for v in str_score.flatten().tolist()],
             "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": comp.h2d_bytes,
                     "d2h_bytes_per_step": comp.d2h_bytes, "ms_per_step": ms_e2e, "steps": n_e2e},

@@ -186,6 +186,19 @@ int cc_compress_layer(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win,
                       int32_t* idx, int32_t* count, const int32_t* free_pages,
                       int32_t* out_page_table, void* ws, size_t ws_bytes, void* stream);
 
+/* Str. Score (Section 5.3, caption of the bug-localization table: "the average fraction of
+ * structurally critical tokens retained across layers and chunks").  For every sequence s and
+ * KV head h: score[s][h] = |{i : prior[idx[h][i]] >= threshold}| / |{j : prior[j] >= threshold}|,
+ * 1 when the sequence has no such token; the average over layers and chunks is the caller's.
+ * idx: device i32 [H_kv][B_tot] as written by cc_topk_select / cc_compress_layer (entries < 0
+ * are skipped); prior: device f32 [N_tot]; score: device f32 [num_seqs][H_kv]; counts: NULL or
+ * device i32 [num_seqs][H_kv][2] receiving (retained critical tokens, critical tokens).
+ * Needs no workspace.  A NaN threshold is CC_ERR_INVALID_ARG; sequences of 2^24 tokens or more
+ * are CC_ERR_UNSUPPORTED (the counts would no longer convert to f32 exactly). */
+int cc_structural_score(cc_ctx* ctx, const cc_layer_desc* desc, const int32_t* idx,
+                        const float* prior, float threshold, float* score, int32_t* counts,
+                        void* stream);
+
 /* Device pointers, inside the workspace last given to cc_compress_layer for `desc`, of the
  * intermediate scores [H_kv][N_tot] and fused values [H_kv][M_tot] (for inspection). */
 int cc_workspace_views(const cc_ctx* ctx, const cc_layer_desc* desc, void* ws,

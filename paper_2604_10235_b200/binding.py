@@ -28,7 +28,8 @@ CC_MAX_SEQS = 64
 
 EXPORTS = ("cc_create", "cc_destroy", "cc_status_string", "cc_last_error", "cc_poll_status",
            "cc_workspace_bytes", "cc_score_window", "cc_fuse_prior_pool", "cc_topk_select",
-           "cc_compact_kv", "cc_compress_layer", "cc_workspace_views", "cc_topk_select_static")
+           "cc_compact_kv", "cc_compress_layer", "cc_workspace_views", "cc_topk_select_static",
+           "cc_structural_score")
 CC_STATIC_SELECT_MAX_ITEMS = 1 << 20
 
 
@@ -89,6 +90,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.cc_fuse_prior_pool.argtypes = [vp, dp, vp, vp, vp, vp]
     lib.cc_topk_select.argtypes = [vp, dp, vp, vp, vp, vp, vp, sz, vp]
     lib.cc_topk_select_static.argtypes = [vp, dp, vp, vp, vp, vp, vp]
+    lib.cc_structural_score.argtypes = [vp, dp, vp, vp, C.c_float, vp, vp, vp]
     lib.cc_compact_kv.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.cc_compress_layer.argtypes = [vp, dp] + [vp] * 10 + [vp, sz, vp]
     lib.cc_workspace_views.argtypes = [vp, dp, vp, C.POINTER(vp), C.POINTER(vp)]
@@ -264,6 +266,13 @@ def cc_compact_kv(ctx: Context, desc: Desc, k, v, idx, k_out, v_out, free_pages=
     ctx.check(ctx.lib.cc_compact_kv(ctx.handle, C.byref(desc.c), _ptr(k), _ptr(v), _ptr(idx),
                                     _ptr(k_out), _ptr(v_out), _ptr(free_pages),
                                     _ptr(out_page_table), _stream(stream)))
+
+
+def cc_structural_score(ctx: Context, desc: Desc, idx, prior, threshold: float, score,
+                        counts=None, stream=None):
+    ctx.check(ctx.lib.cc_structural_score(ctx.handle, C.byref(desc.c), _ptr(idx), _ptr(prior),
+                                          C.c_float(threshold), _ptr(score), _ptr(counts),
+                                          _stream(stream)))
 
 
 def cc_compress_layer(ctx: Context, desc: Desc, q_win, k, v, prior, k_out, v_out, idx, count,

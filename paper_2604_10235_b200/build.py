@@ -11,7 +11,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB_DIR = os.path.join(HERE, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "libcodecomp.so")
-SOURCES = ["api.cu", "score_simt.cu", "score_tc.cu", "fuse_pool.cu", "select.cu", "select_cluster.cu", "compact.cu"]
+SOURCES = ["api.cu", "score_simt.cu", "score_tc.cu", "fuse_pool.cu", "select.cu", "select_cluster.cu", "compact.cu",
+           "str_score.cu"]
 
 
 def nvcc_path() -> str:

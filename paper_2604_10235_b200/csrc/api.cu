@@ -430,6 +430,24 @@ int cc_compress_layer(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win,
   return run_compact(ctx, desc, p, k, v, idx, k_out, v_out, free_pages, out_page_table, stream);
 }
 
+int cc_structural_score(cc_ctx* ctx, const cc_layer_desc* desc, const int32_t* idx,
+                        const float* prior, float threshold, float* score, int32_t* counts,
+                        void* stream) {
+  Plan p;
+  int rc = build_plan(ctx, desc, &p);
+  if (rc != CC_OK) return rc;
+  if (!prior || !score || (!idx && p.bt.b_tot > 0))
+    return fail(ctx, CC_ERR_INVALID_ARG, "NULL tensor pointer");
+  if (threshold != threshold) return fail(ctx, CC_ERR_INVALID_ARG, "threshold is NaN");
+  for (int s = 0; s < p.bt.num_seqs; ++s)
+    if (p.bt.seq[s].n >= (1 << 24))
+      return fail(ctx, CC_ERR_UNSUPPORTED, "sequence %d is too long for exact f32 counts", s);
+  cudaError_t e = launch_str_score(make_launch(ctx, stream), p.bt, p.g, threshold, idx, prior,
+                                   score, counts);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "structural score launch");
+  return CC_OK;
+}
+
 int cc_workspace_views(const cc_ctx* ctx, const cc_layer_desc* desc, void* ws, float** scores,
                        float** fused) {
   Plan p;

@@ -149,4 +149,9 @@ cudaError_t launch_compact(const Launch& L, const BatchTable& bt, const Geometry
                            const void* k, const void* v, const int32_t* idx, void* k_out,
                            void* v_out, const int32_t* free_pages, int32_t* out_page_table);
 
+// fraction of the critical tokens (prior >= threshold) that each head's index list retains
+cudaError_t launch_str_score(const Launch& L, const BatchTable& bt, const Geometry& g,
+                             float threshold, const int32_t* idx, const float* prior,
+                             float* score, int32_t* counts);
+
 }  // namespace cc

@@ -267,3 +267,68 @@ def test_descriptor_validation():
                           torch.zeros(2, 16, dtype=torch.int32, device="cuda"),
                           torch.zeros(2, dtype=torch.int32, device="cuda"), ws=small)
     assert e.value.status == cc.CC_ERR_WORKSPACE
+
+
+# ------------------------------------------------------------------ Str. Score
+@pytest.mark.parametrize("lens,budgets", [((1,), (1,)), ((700,), (64,)), ((4099,), (4099,)),
+                                          ((300, 1, 129, 2050, 64), (30, 1, 12, 205, 6)),
+                                          ((65536,), (2048,))])
+@pytest.mark.parametrize("density,threshold", [(0.07, 0.5), (0.0, 0.5), (1.0, 0.5), (0.3, math.inf)])
+def test_structural_score_matches_oracle(lens, budgets, density, threshold):
+    """Counts bit for bit, fraction as the correctly rounded f32 quotient of the counts."""
+    rng = np.random.Generator(np.random.PCG64(sum(lens) + int(density * 100)))
+    hkv, n_tot, b_tot = 3, sum(lens), sum(min(b, n) for b, n in zip(budgets, lens))
+    prior = (rng.random(n_tot) < density).astype(np.float32) * np.float32(0.75)
+    if density > 0:
+        prior[rng.integers(n_tot)] = 0.5                  # a token exactly at the threshold
+    idx = np.full((hkv, b_tot), -1, dtype=np.int32)
+    off = 0
+    for n, b in zip(lens, budgets):
+        keep = min(b, n)
+        for h in range(hkv):
+            idx[h, off:off + keep] = np.sort(rng.choice(n, size=keep, replace=False))
+        off += keep
+    idx[1, b_tot - 1] = -1                                # padding entries are skipped
+    if len(lens) > 1:
+        d = cc.Desc(hkv, hkv, 4, seq_lens=lens, budgets=budgets)
+    else:
+        d = cc.Desc(hkv, hkv, 4, n=lens[0], budget=budgets[0])
+    score, full_s = guarded((len(lens), hkv), torch.float32, -3.0)
+    counts, full_c = guarded((len(lens), hkv, 2), torch.int32, -3)
+    cc.cc_structural_score(ctx(), d, torch.from_numpy(idx).cuda(), f32_dev(prior), threshold,
+                           score, counts)
+    assert ctx().poll() == 0
+    got_s, got_c = score.cpu().numpy(), counts.cpu().numpy()
+    tok = off = 0
+    for s, (n, b) in enumerate(zip(lens, budgets)):
+        keep = min(b, n)
+        for h in range(hkv):
+            frac, hit, tot = orc.structural_score(idx[h, off:off + keep], prior[tok:tok + n], threshold)
+            assert (got_c[s, h, 0], got_c[s, h, 1]) == (hit, tot)
+            assert got_s[s, h] == np.float32(frac)
+        tok += n
+        off += keep
+    assert guards_intact(full_s, -3.0) and guards_intact(full_c, -3)
+
+
+def test_structural_score_of_the_fused_path_on_tiny():
+    """The retained sets of cc_compress_layer keep every protected token when they fit the budget."""
+    wl = gen.workloads()["tiny"]
+    x = gen.make_layer(wl)
+    d = desc_for(wl, cc.CC_MODE_BF16)
+    hkv, b = wl.n_heads_kv, wl.budget
+    idx = torch.empty((hkv, b), dtype=torch.int32, device="cuda")
+    count = torch.empty((1, hkv), dtype=torch.int32, device="cuda")
+    k_out = torch.empty((b, hkv, 128), dtype=torch.bfloat16, device="cuda")
+    v_out = torch.empty_like(k_out)
+    prior = f32_dev(x.prior)
+    cc.cc_compress_layer(ctx(), d, bf16_dev(x.q_win), bf16_dev(x.k), bf16_dev(x.v), prior, k_out,
+                         v_out, idx, count)
+    score = torch.empty((1, hkv), dtype=torch.float32, device="cuda")
+    cc.cc_structural_score(ctx(), d, idx, prior, wl.force_threshold, score)
+    assert ctx().poll() == 0
+    assert (score.cpu().numpy() == 1.0).all()
+    res = orc.compress_sequence(x.q_win[0], x.k, None, x.prior, hkv, wl.pool_kind, wl.pool_size,
+                                wl.budget, wl.alpha, wl.beta, wl.force_threshold)
+    for h in range(hkv):
+        assert orc.structural_score(res["idx"][h], x.prior, wl.force_threshold)[0] == 1.0
