@@ -35,6 +35,8 @@ unpinned" by the paper, pinned here only by self-consistency tests):
   - the normalisation of the attention term inside ``fuse_prior`` (alpha is a free
     caller-chosen factor);
   - the edge rule of average pooling (zero padding, always divide by the width);
+  - the ``causal`` option of ``window_scores`` (window inside the sequence) is an extension;
+    the paper's window follows the context and needs no mask;
   - ``structural_score`` of a sequence without structurally critical tokens is taken
     as 1 (nothing could be lost); the paper does not say.
 """
@@ -56,7 +58,7 @@ def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------- A1 score
-def window_scores(q_win: np.ndarray, k: np.ndarray, n_heads_kv: int
+def window_scores(q_win: np.ndarray, k: np.ndarray, n_heads_kv: int, causal: bool = False
                   ) -> Tuple[np.ndarray, np.ndarray]:
     """Window attention scores per KV head.
 
@@ -65,9 +67,14 @@ def window_scores(q_win: np.ndarray, k: np.ndarray, n_heads_kv: int
       s_{g,t}(j) = q_{g,t} . k_j / sqrt(d),  A = softmax over the n keys (no mask),
       u_h(j) = sum over the G query heads of KV head h and the w window rows of A,
       lse = log sum_j exp(s) for every (query head, window row).
+    ``causal`` (an extension, not in the paper, whose window follows the context): the window
+    is the last w tokens of the sequence itself, so row t sits at position n - w + t and
+    attends to the keys j <= n - w + t only (A = 0 beyond).
     """
     w, hq, d = q_win.shape
     n = k.shape[0]
+    if causal and n < w:
+        raise ValueError("a causal window needs n >= w")
     g = hq // n_heads_kv
     u = np.zeros((n_heads_kv, n), dtype=np.float64)
     lse = np.zeros((hq, w), dtype=np.float64)
@@ -76,6 +83,9 @@ def window_scores(q_win: np.ndarray, k: np.ndarray, n_heads_kv: int
         for gi in range(g):
             qh = q_win[:, h * g + gi, :]                  # [w][d]
             s = (qh @ kh.T) / math.sqrt(d)                # [w][n]
+            if causal:
+                for t in range(w):
+                    s[t, n - w + t + 1:] = -np.inf
             m = s.max(axis=1, keepdims=True)
             e = np.exp(s - m)
             l = e.sum(axis=1, keepdims=True)
@@ -258,7 +268,7 @@ def compress_sequence(q_bits: np.ndarray, k_bits: np.ndarray, v_bits: Optional[n
                       prior: np.ndarray, n_heads_kv: int, pool_kind: int, pool_size: int,
                       budget: int, alpha: float, beta: float, force_threshold: float,
                       span_ratio: float = 0.0, span_min: int = 0, chunk: int = 1,
-                      stage_dtype=np.float64) -> dict:
+                      stage_dtype=np.float64, causal: bool = False) -> dict:
     """The whole per-layer step for one contiguous sequence.
 
     q_bits [w][H_q][d], k_bits/v_bits [n][H_kv][d] as bf16 bit patterns, prior [n].
@@ -268,7 +278,7 @@ def compress_sequence(q_bits: np.ndarray, k_bits: np.ndarray, v_bits: Optional[n
     q = bf16_bits_to_f64(q_bits)
     k = bf16_bits_to_f64(k_bits)
     n = k.shape[0]
-    u, lse = window_scores(q, k, n_heads_kv)
+    u, lse = window_scores(q, k, n_heads_kv, causal)
     u_s = u.astype(stage_dtype)
     prior_s = np.asarray(prior, dtype=stage_dtype)
     if chunk > 1:

@@ -373,3 +373,57 @@ def test_structural_score_is_one_when_protected_tokens_fit_the_budget():
     res2 = orc.compress_sequence(x.q_win[0], x.k, None, x.prior, wl.n_heads_kv, wl.pool_kind,
                                  wl.pool_size, wl.budget, wl.alpha, wl.beta, float("inf"))
     assert orc.structural_score(res2["idx"][0], x.prior, wl.force_threshold)[0] < 1.0
+
+
+# --------------------------------------------------------------------------- causal window
+def test_causal_window_closed_form_with_identical_keys():
+    """All keys equal: row t spreads its mass evenly over the n - w + t + 1 keys it sees, so
+    u(j) = G * sum over the rows that see j of 1 / (keys the row sees)."""
+    n, w, hq, hkv, d = 40, 6, 4, 2, 128
+    rng = np.random.Generator(np.random.PCG64(5))
+    q = rng.standard_normal((w, hq, d))
+    k = np.broadcast_to(rng.standard_normal((1, hkv, d)), (n, hkv, d)).copy()
+    u, lse = orc.window_scores(q, k, hkv, causal=True)
+    g = hq // hkv
+    want = np.zeros(n)
+    for t in range(w):
+        seen = n - w + t + 1
+        want[:seen] += g / seen
+    np.testing.assert_allclose(u[0], want, rtol=1e-12)
+    np.testing.assert_allclose(u.sum(axis=1), w * g, rtol=1e-12)
+    # lse of row t = s + log(keys seen)
+    s00 = q[0, 0] @ k[0, 0] / math.sqrt(d)
+    np.testing.assert_allclose(lse[0, 0], s00 + math.log(n - w + 1), rtol=1e-12)
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_causal_window_vs_scalar_loops(seed):
+    rng = np.random.Generator(np.random.PCG64(700 + seed))
+    n, w, hq, hkv, d = 11, 4, 2, 1, 128
+    q = rng.standard_normal((w, hq, d))
+    k = rng.standard_normal((n, hkv, d))
+    u, _ = orc.window_scores(q, k, hkv, causal=True)
+    ref = np.zeros(n)
+    for gi in range(hq):
+        for t in range(w):
+            last = n - w + t
+            s = [sum(q[t, gi, c] * k[j, 0, c] for c in range(d)) / math.sqrt(d) for j in range(last + 1)]
+            z = sum(math.exp(x) for x in s)
+            for j in range(last + 1):
+                ref[j] += math.exp(s[j]) / z
+    np.testing.assert_allclose(u[0], ref, rtol=1e-10)
+    # the last key is seen by the last row only; keys before the window are seen by all rows
+    assert u[0, n - 1] <= hq and np.all(u[0] > 0)
+
+
+def test_causal_window_differs_from_unmasked_only_through_the_last_keys():
+    rng = np.random.Generator(np.random.PCG64(77))
+    n, w, hq, hkv, d = 64, 8, 2, 2, 128
+    q, k = rng.standard_normal((w, hq, d)), rng.standard_normal((n, hkv, d))
+    u_c, lse_c = orc.window_scores(q, k, hkv, causal=True)
+    u_f, lse_f = orc.window_scores(q, k, hkv, causal=False)
+    # the last row sees every key: identical log-sum-exp; earlier rows see fewer: smaller
+    np.testing.assert_allclose(lse_c[:, w - 1], lse_f[:, w - 1], rtol=1e-13)
+    assert np.all(lse_c[:, :w - 1] < lse_f[:, :w - 1])
+    with pytest.raises(ValueError):
+        orc.window_scores(q, k[:4], hkv, causal=True)
