@@ -105,6 +105,11 @@ typedef struct cc_layer_desc {
   int32_t page_table_stride;
   int32_t pool_pages;       /* pages in the K/V pool (page ids must be < pool_pages) when page_size > 0 */
   int32_t out_page_table_stride; /* row length of out_page_table (>= ceil(B_s / page_size)) */
+  int32_t causal;           /* 0: the window follows the scored keys and every row attends to all
+                               n_s of them (Section 4.5).  1 (no counterpart in the paper): the
+                               window is the last w tokens of the sequence itself; row t sits at
+                               position n_s - w + t and attends to keys j <= n_s - w + t only.
+                               Needs n_s >= w for every non-empty sequence. */
 } cc_layer_desc;
 
 /* Creates a context on CUDA device `device` (must be compute capability 10.x).  Allocates a

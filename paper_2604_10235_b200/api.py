@@ -22,7 +22,7 @@ def desc_from_workload(wl: gen.Workload, mode: int = cc.CC_MODE_BF16,
               pool_size=wl.pool_size, chunk_size=wl.chunk_size, alpha=wl.alpha, beta=wl.beta,
               force_threshold=wl.force_threshold, span_ratio=wl.span_ratio, span_min=wl.span_min,
               page_size=wl.page_size, page_table=page_table, pool_pages=pool_pages,
-              out_page_table_stride=out_pt_stride)
+              out_page_table_stride=out_pt_stride, causal=wl.causal)
     if wl.seq_lens:
         return cc.Desc(wl.n_heads_q, wl.n_heads_kv, wl.window, seq_lens=wl.lens,
                        budgets=wl.budgets, **kw)

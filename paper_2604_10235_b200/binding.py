@@ -55,6 +55,7 @@ class cc_layer_desc(C.Structure):
         ("page_table", C.c_void_p),
         ("page_table_stride", C.c_int32), ("pool_pages", C.c_int32),
         ("out_page_table_stride", C.c_int32),
+        ("causal", C.c_int32),
     ]
 
 
@@ -160,7 +161,8 @@ class Desc:
                  pool_size: int = 7, chunk_size: int = 1, alpha: float = 1.0, beta: float = 0.0,
                  force_threshold: float = math.inf, span_ratio: float = 0.0, span_min: int = 0,
                  page_size: int = 0, page_table: Optional[torch.Tensor] = None, pool_pages: int = 0,
-                 out_page_table_stride: int = 0, q_strides=None, kv_strides=None,
+                 out_page_table_stride: int = 0, causal: bool = False, q_strides=None,
+                 kv_strides=None,
                  out_strides=(0, 0)):
         c = cc_layer_desc()
         c.n_heads_q, c.n_heads_kv, c.head_dim, c.window = n_heads_q, n_heads_kv, head_dim, window
@@ -193,6 +195,7 @@ class Desc:
             c.page_table_stride = page_table.shape[-1]
         c.pool_pages = pool_pages
         c.out_page_table_stride = out_page_table_stride
+        c.causal = 1 if causal else 0
         self.c = c
 
     # sizes the caller needs to allocate outputs

@@ -105,6 +105,8 @@ int build_plan(cc_ctx* ctx, const cc_layer_desc* d, Plan* p) {
     const int n = d->num_seqs > 0 ? d->seq_lens[s] : d->n;
     const int b = d->num_seqs > 0 ? d->budgets[s] : d->budget;
     if (n < 0 || b < 0) return fail(ctx, CC_ERR_INVALID_ARG, "negative length or budget");
+    if (d->causal && n > 0 && n < d->window)
+      return fail(ctx, CC_ERR_INVALID_ARG, "a causal window needs n >= window (sequence %d)", s);
     SeqInfo& q = bt.seq[s];
     q.n = n;
     q.budget = b;
@@ -139,6 +141,7 @@ int build_plan(cc_ctx* ctx, const cc_layer_desc* d, Plan* p) {
   g.hkv = d->n_heads_kv;
   g.group = group;
   g.window = d->window;
+  g.causal = d->causal != 0;
   g.rows = group * d->window;
   g.q_stride_seq = d->q_stride_seq;
   g.q_stride_row = d->q_stride_row;

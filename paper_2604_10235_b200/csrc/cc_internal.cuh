@@ -46,6 +46,8 @@ struct Geometry {
   int64_t out_stride_tok, out_stride_head;
   const int32_t* page_table;
   int page_table_stride, out_page_table_stride;
+  int causal;      // window rows are the last w tokens of the sequence: row t sees keys <= n - w + t
+  int pad_;
 };
 
 // Device status word: [0] = first error code, [1] = detail (where it happened).

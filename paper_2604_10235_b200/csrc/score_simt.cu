@@ -47,6 +47,8 @@ score_simt_kernel(const __grid_constant__ BatchTable bt, const Geometry g, const
   const float scale = 1.0f / sqrtf((float)kHeadDim);
 
   uint32_t qp[kHeadDim / 2];
+  // last key this row attends to: all of them, or (causal window) its own position n - w + t
+  const int last_key = (g.causal && active) ? sq.n - g.window + r % g.window : sq.n - 1;
   if (active) {
     const int gi = r / g.window, t = r % g.window;
     const uint4* src = reinterpret_cast<const uint4*>(
@@ -125,19 +127,22 @@ score_simt_kernel(const __grid_constant__ BatchTable bt, const Geometry g, const
         float gmax = -INFINITY;
 #pragma unroll
         for (int j = 0; j < kGroup; ++j) {
-          acc[j] = (j0 + j < valid) ? acc[j] * scale : -INFINITY;
+          acc[j] = (j0 + j < valid && base + j0 + j <= last_key) ? acc[j] * scale : -INFINITY;
           gmax = fmaxf(gmax, acc[j]);
         }
-        const float new_max = fmaxf(run_max, gmax);
-        float add = 0.0f;
+        if (gmax > -INFINITY) {          // a causal row may see none of the eight keys
+          const float new_max = fmaxf(run_max, gmax);
+          float add = 0.0f;
 #pragma unroll
-        for (int j = 0; j < kGroup; ++j) add += expf(acc[j] - new_max);
-        run_sum = run_sum * (double)expf(run_max - new_max) + (double)add;
-        run_max = new_max;
+          for (int j = 0; j < kGroup; ++j) add += expf(acc[j] - new_max);
+          run_sum = run_sum * (double)expf(run_max - new_max) + (double)add;
+          run_max = new_max;
+        }
       } else {
 #pragma unroll
         for (int j = 0; j < kGroup; ++j) {
-          float v = (active && j0 + j < valid) ? expf(acc[j] * scale - L) : 0.0f;
+          float v = (active && j0 + j < valid && base + j0 + j <= last_key)
+                        ? expf(acc[j] * scale - L) : 0.0f;
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
           if (lane == 0) colpart[warp][j0 + j] = v;

@@ -34,6 +34,8 @@
 // CC_ERR_TIMEOUT, every role leaves its loop, TMEM is released and the kernel returns.
 #include <string.h>
 
+#include <type_traits>
+
 #include "cc_internal.cuh"
 
 #ifndef CC_POLY_EVERY
@@ -367,7 +369,9 @@ __device__ __forceinline__ int cta_of_tile(int t, const TcParams& P) {
 }
 
 // ------------------------------------------------------------------ the kernel
-template <int PASS>
+// CAUSAL instantiations carry the masked copies of the epilogue loops; the others have none of
+// that code.
+template <int PASS, bool CAUSAL>
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ Geometry g,
                 const __grid_constant__ TcParams P, const __grid_constant__ CUtensorMap q_map,
@@ -728,8 +732,20 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
 #pragma unroll
             for (int rb = 1; rb < 4; ++rb) if (rb == sub) { m_run = run_m[rb]; l_run = run_l[rb]; }
           }
+          // keys of the tile this row attends to: all valid ones, or (causal window) those up
+          // to the row's own position n - w + t
+          // (the masked form is a copy of the loop of its own, so that the common one stays lean)
+          const bool masked_tile = CAUSAL && key0 + kTileKeys > n_cur - g.window + 1;
+          auto drain = [&](auto masked) {
+          constexpr bool kMasked = decltype(masked)::value;
+          int valid_r = valid;
+          if (kMasked) {
+            const int t_row = (sub * 128 + row_in_tile) / g.group;
+            if (t_row < g.window) valid_r = min(valid, n_cur - g.window + t_row + 1 - key0);
+          }
 #pragma unroll 1
           for (int cc0 = 0; cc0 < kTileKeys; cc0 += 32) {
+            if (kMasked) __syncwarp();            // rows of a masked tile skip different chunks
             tmem_ld32(acc_addr + (uint32_t)cc0, v);
             tmem_wait_ld();
             if (cc0 + 32 == kTileKeys) {             // last read of the buffer: hand it back
@@ -737,11 +753,11 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
               __syncwarp();
               if (lane == 0) mbar_arrive(empty_bar);
             }
-            if (cc0 >= valid) continue;
-            if (cc0 + 32 > valid) {
+            if (cc0 >= valid_r) continue;
+            if (cc0 + 32 > valid_r) {
 #pragma unroll
               for (int i = 0; i < 32; ++i)
-                if (cc0 + i >= valid) v[i] = 0xc61c4000u;    // -1e4: its exponential underflows to 0
+                if (cc0 + i >= valid_r) v[i] = 0xc61c4000u;  // -1e4: its exponential underflows to 0
             }
             // The reference of the exponentials only has to be near the row maximum, not equal
             // to it: it is replaced when a value lies more than 2^64 above it.
@@ -753,6 +769,8 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
             }
             exp_accumulate<false, 32>(v, c2, pack2(-m_run, -m_run), nullptr, acc);
           }
+          };
+          if (CAUSAL && masked_tile) drain(std::true_type{}); else drain(std::false_type{});
           l_run += acc_total(acc);
           if (rotating) {
 #pragma unroll
@@ -766,10 +784,22 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
           const int c0 = sub * P.sub_cols;
           const int nc = min(P.sub_cols, P.rows_pad - c0);        // multiple of 16
           const float* nl = misc->neg_lc + c0;
+          // causal window: key j is seen by the rows t >= j - (n - w), i.e. by the columns
+          // from G * (j - n + w) on; the columns before it contribute nothing
+          const bool masked_tile = CAUSAL && key0 + kTileKeys > n_cur - g.window + 1;
+          auto drain = [&](auto masked) {
+          constexpr bool kMasked = decltype(masked)::value;
+          const int first_col = kMasked ? g.group * (key0 + row_in_tile - n_cur + g.window) : 0;
 #pragma unroll 1
           for (int cc0 = 0; cc0 < nc; cc0 += 32) {
+            if (kMasked) __syncwarp();
             tmem_ld32(acc_addr + (uint32_t)cc0, v);               // stays inside the 128-column buffer
             tmem_wait_ld();
+            if (kMasked && first_col > c0 + cc0) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (c0 + cc0 + i < first_col) v[i] = 0xc61c4000u;   // -1e4: exponential ~ 0
+            }
             if (cc0 + 32 >= nc) {
               tc_fence_before();
               __syncwarp();
@@ -778,6 +808,8 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
             if (cc0 + 32 <= nc) exp_accumulate<true, 32>(v, c2, 0ull, nl + cc0, acc);
             else                exp_accumulate<true, 16>(v, c2, 0ull, nl + cc0, acc);
           }
+          };
+          if (CAUSAL && masked_tile) drain(std::true_type{}); else drain(std::false_type{});
           u_acc = acc_total(acc);
         }
       }
@@ -911,24 +943,24 @@ cudaError_t launch_score_tc(const Launch& L, const BatchTable& bt, const Geometr
     if (r != CUDA_SUCCESS) { *drv_err = (int)r; return cudaErrorUnknown; }
   }
 
+  auto pass1 = g.causal ? score_tc_kernel<1, true> : score_tc_kernel<1, false>;
+  auto pass2 = g.causal ? score_tc_kernel<2, true> : score_tc_kernel<2, false>;
   cudaError_t e;
-  e = cudaFuncSetAttribute(score_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)pl.smem_bytes);
+  e = cudaFuncSetAttribute(pass1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(score_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)pl.smem_bytes);
+  e = cudaFuncSetAttribute(pass2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes);
   if (e != cudaSuccess) return e;
 
   P.n_sub = (P.rows_pad + 127) / 128;
   P.sub_cols = 0;
-  e = launch_pdl(score_tc_kernel<1>, dim3(P.grid), dim3(kThreads), pl.smem_bytes, L.stream, 1, bt, g, P,
-                 q_map, k_map, L.status);
+  e = launch_pdl(pass1, dim3(P.grid), dim3(kThreads), pl.smem_bytes, L.stream, 1, bt, g, P, q_map,
+                 k_map, L.status);
   if (e != cudaSuccess) return e;
 
   P.n_sub = (P.rows_pad + 127) / 128;
   P.sub_cols = ((P.rows_pad + P.n_sub - 1) / P.n_sub + 15) / 16 * 16;
-  return launch_pdl(score_tc_kernel<2>, dim3(P.grid), dim3(kThreads), pl.smem_bytes, L.stream, 1, bt, g,
-                    P, q_map, k_map, L.status);
+  return launch_pdl(pass2, dim3(P.grid), dim3(kThreads), pl.smem_bytes, L.stream, 1, bt, g, P, q_map,
+                    k_map, L.status);
 }
 
 }  // namespace cc

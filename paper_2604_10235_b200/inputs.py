@@ -52,6 +52,7 @@ class Workload:
     force_threshold: float = 0.5     # prior >= threshold -> forced retention
     span_ratio: float = 0.0          # 0 = no cap on forced tokens
     span_min: int = 16
+    causal: bool = False             # window = last w tokens of the sequence itself (masked)
 
     @property
     def group(self) -> int:

@@ -63,7 +63,7 @@ def check_layer(wl, x, mode, tol):
         prior = x.prior[lo:lo + n]
         ref = orc.compress_sequence(x.q_win[s], k_s, v_s, prior, wl.n_heads_kv, wl.pool_kind,
                                     wl.pool_size, b, wl.alpha, wl.beta, wl.force_threshold,
-                                    wl.span_ratio, wl.span_min, chunk)
+                                    wl.span_ratio, wl.span_min, chunk, causal=wl.causal)
         assert_scores_close(got["scores"][:, lo:lo + n], ref["scores"], rows, n, tol)
         m = len(ref["item_prior"])
         forced_items = ref["item_prior"].astype(np.float32) >= np.float32(wl.force_threshold)
@@ -121,6 +121,12 @@ def test_paper_setting_avg_pool(mode, tol):
 def test_weighted_prior_mode(mode, tol):
     from dataclasses import replace
     wl = replace(gen.workloads()["tiny"], alpha=0.06 / (32 * 4), beta=1.0, force_threshold=float("inf"))
+    check_layer(wl, gen.make_layer(wl), mode, tol)
+
+
+@pytest.mark.parametrize("mode,tol", MODES)
+def test_causal_window_fused_path(mode, tol):
+    wl = gen.Workload("causal", 33, 1, 8, 2, 128, 32, gen.POOL_MAX, 7, 200, n=1500, causal=True)
     check_layer(wl, gen.make_layer(wl), mode, tol)
 
 

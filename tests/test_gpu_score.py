@@ -32,7 +32,7 @@ def check_against_oracle(wl, x, mode, tol):
     for s, n in enumerate(wl.lens):
         k_s, _ = seq_kv(x, s)
         ref, lse_ref = orc.window_scores(orc.bf16_bits_to_f64(x.q_win[s]), orc.bf16_bits_to_f64(k_s),
-                                         wl.n_heads_kv)
+                                         wl.n_heads_kv, causal=wl.causal)
         lo = int(x.tok_offsets[s])
         assert_scores_close(u[:, lo:lo + n], ref, rows, n, tol)
         np.testing.assert_allclose(lse[s], lse_ref, atol=20 * tol, rtol=0)
@@ -90,3 +90,31 @@ def test_scores_large_logits_do_not_overflow(mode, tol):
     q = orc.bf16_bits_to_f64(x.q_win).astype(np.float32) * 12.0       # logits of order +-150
     x.q_win = gen.f32_to_bf16_bits(q)
     check_against_oracle(wl, x, mode, tol)
+
+
+# ------------------------------------------------------------------ causal in-sequence window
+@pytest.mark.parametrize("mode,tol", MODES)
+@pytest.mark.parametrize("n,w,hq,hkv", [(32, 32, 8, 2), (33, 32, 8, 2), (127, 16, 4, 1), (128, 64, 4, 1),
+                                        (129, 64, 32, 8), (300, 128, 4, 1), (1000, 64, 28, 4),
+                                        (4099, 32, 8, 2), (200, 3, 6, 2), (512, 128, 8, 2)])
+def test_scores_causal_window(mode, tol, n, w, hq, hkv):
+    """The window is the last w tokens of the sequence: row t attends to keys <= n - w + t."""
+    wl = gen.Workload("causal", 24, 1, hq, hkv, 128, w, gen.POOL_MAX, 7, 1, n=n, causal=True)
+    check_against_oracle(wl, gen.make_layer(wl, layer=n + w, with_v=False), mode, tol)
+
+
+@pytest.mark.parametrize("mode,tol", MODES)
+@pytest.mark.parametrize("page", [0, 16])
+def test_scores_causal_ragged_batch(mode, tol, page):
+    wl = gen.Workload("causal_ragged", 25, 1, 8, 2, 128, 16, gen.POOL_MAX, 7, 0,
+                      seq_lens=(300, 16, 129, 2050, 64), budget_frac=0.1, page_size=page, causal=True)
+    check_against_oracle(wl, gen.make_layer(wl, with_v=False), mode, tol)
+
+
+def test_causal_window_shorter_than_the_window_is_rejected():
+    d = cc.Desc(8, 2, 32, n=20, budget=4, causal=True)
+    scores = torch.empty((2, 20), device="cuda")
+    q = torch.empty((1, 32, 8, 128), dtype=torch.bfloat16, device="cuda")
+    k = torch.empty((20, 2, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(cc.CodecompError):
+        cc.cc_score_window(ctx(), d, q, k, scores, None)
