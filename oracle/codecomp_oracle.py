@@ -25,6 +25,11 @@ What each function follows:
                         (remaining capacity filled by top-ranked attention scores).
 * ``compact_kv``      - the retained K/V rows in original order (Section 4.6: chunks
                         keep their original position indices).
+* ``plan_budgets``    - Section 4.3 "Structure-Aware Budget Allocation": normalised chunk
+                        scores, capacity multipliers and the per-chunk token budgets B_i.
+* ``select_spans``    - Section 4.4 "Span selection under budget": protected spans first,
+                        the others greedily by score within B^span; returns the tokens
+                        they cover (the set P_i that "Token-level protection" starts from).
 * ``structural_score`` - Section 5.3, caption of the bug-localization table: the fraction
                         of structurally critical tokens that a retained set contains
                         (the table averages it over layers and chunks; the average is
@@ -37,6 +42,9 @@ unpinned" by the paper, pinned here only by self-consistency tests):
   - the edge rule of average pooling (zero padding, always divide by the width);
   - the ``causal`` option of ``window_scores`` (window inside the sequence) is an extension;
     the paper's window follows the context and needs no mask;
+  - ``select_spans``: "added greedily until the span budget is exhausted" is read as: spans
+    are taken whole, in rank order (score descending, earlier start first), while the
+    tokens covered so far are fewer than B^span, so the last span taken may overshoot it;
   - ``structural_score`` of a sequence without structurally critical tokens is taken
     as 1 (nothing could be lost); the paper does not say.
 """
@@ -231,6 +239,55 @@ def compact_kv(k_bits: np.ndarray, v_bits: np.ndarray, idx: Sequence[np.ndarray]
     k_out = [k_bits[np.asarray(ix, dtype=np.int64), h, :] for h, ix in enumerate(idx)]
     v_out = [v_bits[np.asarray(ix, dtype=np.int64), h, :] for h, ix in enumerate(idx)]
     return k_out, v_out
+
+
+# --------------------------------------------------------------------------- budget planner
+def plan_budgets(sigma: Sequence[float], lens: Sequence[int], r: float, r_max: float,
+                 m_min: float, m_max: float, eps: float) -> Tuple[np.ndarray, np.ndarray]:
+    """Per-chunk token budgets from the chunk-level structural scores (Section 4.3).
+
+    s~_i = 0.5 if all scores are equal, else (sigma_i - min) / max(eps, max - min);
+    m_i = m_min + (m_max - m_min) * clip(s~_i, 0, 1);  B_i = floor(|C_i| * min(r_max, r * m_i)).
+    Everything in fp64, in exactly this operation order.  Returns (B [int64], m [float64])."""
+    sig = np.asarray(sigma, dtype=np.float64)
+    budgets = np.zeros(len(sig), dtype=np.int64)
+    mult = np.zeros(len(sig), dtype=np.float64)
+    if len(sig) == 0:
+        return budgets, mult
+    lo, hi = float(sig.min()), float(sig.max())
+    for i, (sg, length) in enumerate(zip(sig, lens)):
+        st = 0.5 if hi == lo else (float(sg) - lo) / max(float(eps), hi - lo)
+        st = min(1.0, max(0.0, st))
+        mult[i] = float(m_min) + (float(m_max) - float(m_min)) * st
+        # same 1e-9 nudge as span_budget: products that are integers on paper stay integers
+        budgets[i] = math.floor(float(length) * min(float(r_max), float(r) * mult[i]) + 1e-9)
+    return budgets, mult
+
+
+def select_spans(starts: Sequence[int], ends: Sequence[int], scores: Sequence[float],
+                 protected: Sequence[bool], n: int, budget: int, span_ratio: float,
+                 span_min: int) -> Tuple[np.ndarray, List[int]]:
+    """Tokens covered by the spans selected under the span budget (Section 4.4).
+
+    Spans are half-open token ranges [start, end) inside [0, n).  Protected spans are all
+    taken; the others follow in rank order (score descending, earlier start, lower index) while
+    fewer than B^span = min(B, max(B_min, floor(rho * B))) tokens are covered.
+    Returns (mask [n] of covered tokens, indices of the spans taken in the order taken)."""
+    cap = span_budget(budget, span_ratio, span_min) if span_ratio > 0 else budget
+    mask = np.zeros(n, dtype=bool)
+    taken: List[int] = []
+    for i in range(len(starts)):
+        if protected[i]:
+            mask[starts[i]:ends[i]] = True
+            taken.append(i)
+    rest = [i for i in range(len(starts)) if not protected[i]]
+    rest.sort(key=lambda i: (-float(np.float32(scores[i])), starts[i], i))
+    for i in rest:
+        if int(mask.sum()) >= cap:
+            break
+        mask[starts[i]:ends[i]] = True
+        taken.append(i)
+    return mask, taken
 
 
 # --------------------------------------------------------------------------- Str. Score

@@ -427,3 +427,80 @@ def test_causal_window_differs_from_unmasked_only_through_the_last_keys():
     assert np.all(lse_c[:, :w - 1] < lse_f[:, :w - 1])
     with pytest.raises(ValueError):
         orc.window_scores(q, k[:4], hkv, causal=True)
+
+
+# --------------------------------------------------------------------------- budget planner
+def test_plan_budgets_hand_values():
+    """Section 4.3, worked by hand with the appendix's multiplier range [0.5, 1.5]:
+    sigma = (.2, .5, .8) -> s~ = (0, .5, 1) -> m = (.5, 1, 1.5) -> ratios (.2, .4, .6)."""
+    b, m = orc.plan_budgets([0.2, 0.5, 0.8], [1000, 2000, 4096], 0.4, 1.0, 0.5, 1.5, 1e-6)
+    np.testing.assert_allclose(m, [0.5, 1.0, 1.5], rtol=1e-12)
+    assert b.tolist() == [200, 800, 2457]                     # floor(2457.6)
+    # equal scores: s~ = 0.5 for everyone, the multiplier is the middle of the range
+    b, m = orc.plan_budgets([0.3, 0.3], [512, 4096], 0.6, 1.0, 0.5, 1.5, 1e-6)
+    assert m.tolist() == [1.0, 1.0] and b.tolist() == [307, 2457]
+    # the ratio is capped at r_max: 0.8 * 1.5 = 1.2 -> 1.0 -> the whole chunk
+    b, _ = orc.plan_budgets([0.0, 1.0], [100, 100], 0.8, 1.0, 0.5, 1.5, 1e-6)
+    assert b.tolist() == [40, 100]
+    # a spread below eps is divided by eps, not by itself
+    _, m = orc.plan_budgets([0.5, 0.5 + 1e-9], [10, 10], 0.5, 1.0, 0.5, 1.5, 1e-6)
+    np.testing.assert_allclose(m, [0.5, 0.5 + 1e-3], rtol=1e-6)
+    assert orc.plan_budgets([], [], 0.4, 1.0, 0.5, 1.5, 1e-6)[0].size == 0
+
+
+def test_plan_budgets_invariants():
+    rng = np.random.Generator(np.random.PCG64(31))
+    sigma = rng.random(50)
+    lens = np.full(50, 3000)
+    b, m = orc.plan_budgets(sigma, lens, 0.4, 0.9, 0.5, 1.5, 1e-6)
+    order = np.argsort(sigma)
+    assert np.all(np.diff(b[order]) >= 0)                      # more structure, more capacity
+    assert m.min() == 0.5 and m.max() == 1.5                   # the extremes map to the range ends
+    assert np.all(b <= np.floor(lens * 0.9 + 1e-9)) and np.all(b >= np.floor(lens * 0.4 * 0.5))
+
+
+def test_select_spans_hand_case():
+    """Section 4.4: B = 10, rho = 0.5, B_min = 2 -> B^span = 5.  The protected span (3 tokens)
+    comes first; of the two spans with score .9 the earlier one follows (7 covered >= 5: stop)."""
+    starts, ends = [0, 5, 10, 20], [3, 9, 12, 25]
+    mask, taken = orc.select_spans(starts, ends, [0.2, 0.9, 0.9, 0.5], [True, False, False, False],
+                                   30, 10, 0.5, 2)
+    assert taken == [0, 1]
+    assert np.flatnonzero(mask).tolist() == [0, 1, 2, 5, 6, 7, 8]
+    # protected spans are taken even beyond the span budget; nothing else follows then
+    mask, taken = orc.select_spans(starts, ends, [0.2, 0.9, 0.9, 0.5], [True, False, False, True],
+                                   30, 10, 0.5, 2)
+    assert taken == [0, 3] and int(mask.sum()) == 8
+    # overlapping spans count their union
+    mask, taken = orc.select_spans([0, 2], [4, 6], [0.5, 0.4], [False, False], 10, 10, 1.0, 1)
+    assert taken == [0, 1] and int(mask.sum()) == 6
+    assert orc.select_spans([], [], [], [], 5, 3, 0.5, 1)[1] == []
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_select_spans_properties(seed):
+    rng = np.random.Generator(np.random.PCG64(400 + seed))
+    n, k = 200, 25
+    starts = rng.integers(0, n - 10, size=k)
+    ends = starts + rng.integers(1, 10, size=k)
+    scores = rng.integers(0, 5, size=k) / 4.0                  # many ties
+    prot = rng.random(k) < 0.15
+    budget, rho, bmin = 60, 0.5, 16
+    cap = orc.span_budget(budget, rho, bmin)
+    mask, taken = orc.select_spans(starts, ends, scores, prot, n, budget, rho, bmin)
+    n_prot = int(prot.sum())
+    assert taken[:n_prot] == [i for i in range(k) if prot[i]]
+    rest = taken[n_prot:]
+    rank = sorted((i for i in range(k) if not prot[i]), key=lambda i: (-scores[i], starts[i], i))
+    assert rest == rank[:len(rest)]                            # a prefix of the rank order
+    cover = np.zeros(n, dtype=bool)
+    for i in taken[:-1] if rest else taken:
+        cover[starts[i]:ends[i]] = True
+    if rest:
+        assert cover.sum() < cap                               # the last one was still needed
+    if len(rest) < len(rank):
+        assert mask.sum() >= cap                               # stopped because the budget is used
+    want = np.zeros(n, dtype=bool)
+    for i in taken:
+        want[starts[i]:ends[i]] = True
+    assert np.array_equal(mask, want)
