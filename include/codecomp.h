@@ -204,6 +204,41 @@ int cc_structural_score(cc_ctx* ctx, const cc_layer_desc* desc, const int32_t* i
                         const float* prior, float threshold, float* score, int32_t* counts,
                         void* stream);
 
+/* ---- host-side planning (no GPU work, no context; all pointers are HOST memory) ----------- */
+
+/* Section 4.3 "Structure-Aware Budget Allocation", with the appendix's multiplier range
+ * [0.5, 1.5] as the usual m_min, m_max. */
+typedef struct cc_budget_params {
+  double r;        /* base compression ratio */
+  double r_max;    /* cap on a chunk's ratio */
+  double m_min;    /* capacity multiplier of the structurally least important chunk */
+  double m_max;    /* ... of the most important one (>= m_min) */
+  double eps;      /* floor of the score spread in the normalisation (> 0) */
+} cc_budget_params;
+
+/* Per-chunk budgets from the chunk-level structural scores sigma_i:
+ *   s~_i = 0.5 if all sigma are equal, else (sigma_i - min) / max(eps, max - min);
+ *   m_i = m_min + (m_max - m_min) * clip(s~_i, 0, 1);
+ *   budgets[i] = floor(lens[i] * min(r_max, r * m_i)), never above lens[i];
+ * evaluated in double precision in this order.  multipliers (nullable) receives m_i.
+ * The budgets are what cc_layer_desc.budgets takes when every chunk is a sequence of a batch.
+ * NaN scores, negative lengths or parameters out of range: CC_ERR_INVALID_ARG. */
+int cc_plan_budgets(const double* sigma, const int32_t* lens, int32_t num_chunks,
+                    const cc_budget_params* p, int32_t* budgets, double* multipliers);
+
+/* Section 4.4 "Span selection under budget" for one chunk of n tokens with budget B: spans are
+ * half-open token ranges [starts[i], ends[i]); all protected spans (signatures, query-matched)
+ * are taken; the others follow in rank order (score descending, then earlier start, then lower
+ * index), each taken whole, while fewer than B_span = min(B, max(span_min, floor(span_ratio *
+ * B))) tokens are covered (span_ratio <= 0: B_span = B).  prior_mask [n] receives 1.0 for the
+ * covered tokens and 0.0 elsewhere: given as `prior` with force_threshold <= 1 it makes them the
+ * protected set P_i of the selection ("Token-level protection").  taken (nullable, room for
+ * num_spans) receives the indices of the spans in the order taken, num_taken their number. */
+int cc_select_spans(const int32_t* starts, const int32_t* ends, const float* scores,
+                    const uint8_t* is_protected, int32_t num_spans, int32_t n, int32_t budget,
+                    double span_ratio, int32_t span_min, float* prior_mask, int32_t* taken,
+                    int32_t* num_taken);
+
 /* Device pointers, inside the workspace last given to cc_compress_layer for `desc`, of the
  * intermediate scores [H_kv][N_tot] and fused values [H_kv][M_tot] (for inspection). */
 int cc_workspace_views(const cc_ctx* ctx, const cc_layer_desc* desc, void* ws,

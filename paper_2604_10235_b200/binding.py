@@ -29,7 +29,7 @@ CC_MAX_SEQS = 64
 EXPORTS = ("cc_create", "cc_destroy", "cc_status_string", "cc_last_error", "cc_poll_status",
            "cc_workspace_bytes", "cc_score_window", "cc_fuse_prior_pool", "cc_topk_select",
            "cc_compact_kv", "cc_compress_layer", "cc_workspace_views", "cc_topk_select_static",
-           "cc_structural_score")
+           "cc_structural_score", "cc_plan_budgets", "cc_select_spans")
 CC_STATIC_SELECT_MAX_ITEMS = 1 << 20
 
 
@@ -93,6 +93,9 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.cc_topk_select_static.argtypes = [vp, dp, vp, vp, vp, vp, vp]
     lib.cc_structural_score.argtypes = [vp, dp, vp, vp, C.c_float, vp, vp, vp]
     lib.cc_compact_kv.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.cc_plan_budgets.argtypes = [vp, vp, C.c_int32, C.POINTER(cc_budget_params), vp, vp]
+    lib.cc_select_spans.argtypes = [vp, vp, vp, vp, C.c_int32, C.c_int32, C.c_int32, C.c_double,
+                                    C.c_int32, vp, vp, vp]
     lib.cc_compress_layer.argtypes = [vp, dp] + [vp] * 10 + [vp, sz, vp]
     lib.cc_workspace_views.argtypes = [vp, dp, vp, C.POINTER(vp), C.POINTER(vp)]
     for name in EXPORTS:
@@ -101,6 +104,11 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     if path == _build.LIB_PATH:
         _LIB = lib
     return lib
+
+
+class cc_budget_params(C.Structure):
+    _fields_ = [("r", C.c_double), ("r_max", C.c_double), ("m_min", C.c_double),
+                ("m_max", C.c_double), ("eps", C.c_double)]
 
 
 class Context:
@@ -276,6 +284,46 @@ def cc_structural_score(ctx: Context, desc: Desc, idx, prior, threshold: float, 
     ctx.check(ctx.lib.cc_structural_score(ctx.handle, C.byref(desc.c), _ptr(idx), _ptr(prior),
                                           C.c_float(threshold), _ptr(score), _ptr(counts),
                                           _stream(stream)))
+
+
+def _host(a: np.ndarray):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def cc_plan_budgets(sigma, lens, r: float, r_max: float = 1.0, m_min: float = 0.5,
+                    m_max: float = 1.5, eps: float = 1e-6, lib=None):
+    """Host call (no GPU): per-chunk budgets and capacity multipliers (numpy arrays)."""
+    lib = lib or load_library()
+    sigma = np.ascontiguousarray(sigma, dtype=np.float64)
+    lens = np.ascontiguousarray(lens, dtype=np.int32)
+    budgets = np.zeros(len(sigma), dtype=np.int32)
+    mult = np.zeros(len(sigma), dtype=np.float64)
+    p = cc_budget_params(r, r_max, m_min, m_max, eps)
+    rc = lib.cc_plan_budgets(_host(sigma), _host(lens), len(sigma), C.byref(p), _host(budgets),
+                             _host(mult))
+    if rc != CC_OK:
+        raise CodecompError(rc, lib.cc_status_string(rc).decode())
+    return budgets, mult
+
+
+def cc_select_spans(starts, ends, scores, protected, n: int, budget: int, span_ratio: float,
+                    span_min: int, lib=None):
+    """Host call (no GPU): prior mask [n] of the tokens covered by the selected spans and the
+    indices of the spans in the order taken."""
+    lib = lib or load_library()
+    starts = np.ascontiguousarray(starts, dtype=np.int32)
+    ends = np.ascontiguousarray(ends, dtype=np.int32)
+    scores = np.ascontiguousarray(scores, dtype=np.float32)
+    prot = np.ascontiguousarray(protected, dtype=np.uint8)
+    mask = np.zeros(max(n, 1), dtype=np.float32)
+    taken = np.zeros(max(len(starts), 1), dtype=np.int32)
+    count = C.c_int32(0)
+    rc = lib.cc_select_spans(_host(starts), _host(ends), _host(scores), _host(prot), len(starts), n,
+                             budget, span_ratio, span_min, _host(mask), _host(taken),
+                             C.cast(C.byref(count), C.c_void_p))
+    if rc != CC_OK:
+        raise CodecompError(rc, lib.cc_status_string(rc).decode())
+    return mask[:n], taken[:count.value]
 
 
 def cc_compress_layer(ctx: Context, desc: Desc, q_win, k, v, prior, k_out, v_out, idx, count,
