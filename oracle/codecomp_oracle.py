@@ -25,6 +25,9 @@ What each function follows:
                         (remaining capacity filled by top-ranked attention scores).
 * ``compact_kv``      - the retained K/V rows in original order (Section 4.6: chunks
                         keep their original position indices).
+* ``ppl_chunk_scores`` / ``select_chunks`` - Section 4.1 "Query-Conditioned Chunk Selection":
+                        mean negative log-likelihood of the query tokens given each chunk,
+                        and the k chunks with the lowest value.
 * ``plan_budgets``    - Section 4.3 "Structure-Aware Budget Allocation": normalised chunk
                         scores, capacity multipliers and the per-chunk token budgets B_i.
 * ``select_spans``    - Section 4.4 "Span selection under budget": protected spans first,
@@ -239,6 +242,31 @@ def compact_kv(k_bits: np.ndarray, v_bits: np.ndarray, idx: Sequence[np.ndarray]
     k_out = [k_bits[np.asarray(ix, dtype=np.int64), h, :] for h, ix in enumerate(idx)]
     v_out = [v_bits[np.asarray(ix, dtype=np.int64), h, :] for h, ix in enumerate(idx)]
     return k_out, v_out
+
+
+# --------------------------------------------------------------------------- chunk selection
+def ppl_chunk_scores(logits: np.ndarray, targets: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Query-conditioned perplexity score of every chunk (Section 4.1).
+
+    logits [chunks][T][V] (any float type, used as fp64): row (i, t) holds the model's
+    next-token logits for query position t when the context is prefix + chunk i;
+    targets [T]: the query tokens q_t.  -log p(q_t | ...) = logsumexp(row) - row[q_t].
+    Returns (s_ppl [chunks] = mean over t, nll [chunks][T])."""
+    x = np.asarray(logits, dtype=np.float64)
+    m = x.max(axis=2, keepdims=True)
+    lse = (m + np.log(np.exp(x - m).sum(axis=2, keepdims=True)))[:, :, 0]
+    tgt = np.take_along_axis(x, np.asarray(targets, dtype=np.int64)[None, :, None], axis=2)[:, :, 0]
+    nll = lse - tgt
+    return nll.mean(axis=1), nll
+
+
+def select_chunks(scores: np.ndarray, k: int) -> np.ndarray:
+    """Indices of the k chunks with the lowest score, best first; equal scores: lower index
+    first (the paper is silent on ties); NaN ranks last."""
+    s = np.asarray(scores, dtype=np.float64)
+    key = np.where(np.isnan(s), np.inf, s)
+    order = sorted(range(len(s)), key=lambda i: (key[i], i))
+    return np.asarray(order[:max(0, min(k, len(s)))], dtype=np.int64)
 
 
 # --------------------------------------------------------------------------- budget planner

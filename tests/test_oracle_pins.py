@@ -504,3 +504,52 @@ def test_select_spans_properties(seed):
     for i in taken:
         want[starts[i]:ends[i]] = True
     assert np.array_equal(mask, want)
+
+
+# --------------------------------------------------------------------------- chunk selection
+def test_ppl_scores_closed_forms():
+    """Section 4.1.  Uniform logits: p = 1/V for every token, so the score is log V.  One-hot
+    logits of height a on the target: -log p = log(1 + (V - 1) e^-a)."""
+    chunks, t, v = 3, 5, 11
+    tgt = np.array([0, 3, 10, 3, 7])
+    s, nll = orc.ppl_chunk_scores(np.zeros((chunks, t, v)), tgt)
+    np.testing.assert_allclose(s, math.log(v), rtol=1e-14)
+    a = 2.5
+    x = np.zeros((1, t, v))
+    x[0, np.arange(t), tgt] = a
+    s, nll = orc.ppl_chunk_scores(x, tgt)
+    np.testing.assert_allclose(nll, math.log(1 + (v - 1) * math.exp(-a)), rtol=1e-13)
+    # adding a constant to a row changes nothing; the score is the mean over the query tokens
+    y = x + np.arange(t)[None, :, None] * 100.0
+    np.testing.assert_allclose(orc.ppl_chunk_scores(y, tgt)[1], nll, rtol=1e-12)
+    x[0, 0, :] = 0.0
+    s2, nll2 = orc.ppl_chunk_scores(x, tgt)
+    np.testing.assert_allclose(s2[0], (math.log(v) + (t - 1) * nll[0, 1]) / t, rtol=1e-13)
+
+
+def test_ppl_scores_vs_scalar_loops():
+    rng = np.random.Generator(np.random.PCG64(12))
+    x = rng.standard_normal((2, 3, 7)) * 3
+    tgt = np.array([6, 0, 2])
+    s, nll = orc.ppl_chunk_scores(x, tgt)
+    for i in range(2):
+        acc = 0.0
+        for t in range(3):
+            z = sum(math.exp(x[i, t, j]) for j in range(7))
+            want = -math.log(math.exp(x[i, t, tgt[t]]) / z)
+            assert abs(nll[i, t] - want) < 1e-12
+            acc += want
+        assert abs(s[i] - acc / 3) < 1e-12
+
+
+def test_select_chunks_lowest_first_with_ties():
+    s = np.array([2.0, 0.5, 2.0, 0.5, np.nan, 1.0])
+    assert orc.select_chunks(s, 3).tolist() == [1, 3, 5]
+    assert orc.select_chunks(s, 6).tolist() == [1, 3, 5, 0, 2, 4]
+    assert orc.select_chunks(s, 9).tolist() == [1, 3, 5, 0, 2, 4]
+    assert orc.select_chunks(s, 0).tolist() == []
+    rng = np.random.Generator(np.random.PCG64(3))
+    r = rng.integers(0, 6, size=40).astype(np.float64)
+    got = orc.select_chunks(r, 10)
+    assert np.array_equal(np.sort(r)[:10], r[got])           # against the library sort
+    assert all(r[a] < r[b] or (r[a] == r[b] and a < b) for a, b in zip(got[:-1], got[1:]))
