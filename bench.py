@@ -322,6 +322,7 @@ def run_ours(args, wl):
     ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / n_e2e
     e2e_value = sharding.job_throughput(work["tokens"], world, ms_e2e)
 
+    aux = chunk_scoring_bandwidth(ctx, peaks) if rank == 0 and world == 1 else None
     if rank == 0:
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
@@ -352,6 +353,7 @@ def run_ours(args, wl):
                          "select": stage_ms[2] * 1e3, "compact": stage_ms[3] * 1e3,
                          "str_score_diagnostic": stage_ms[4] * 1e3},
             "str_score": [round(float(v), 4) for v in str_score.flatten().tolist()],
+            "chunk_scoring": aux,
             "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": comp.h2d_bytes,
                     "d2h_bytes_per_step": comp.d2h_bytes, "ms_per_step": ms_e2e, "steps": n_e2e},
@@ -362,6 +364,40 @@ def run_ours(args, wl):
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def chunk_scoring_bandwidth(ctx, peaks):
+    """Not part of a step: the chunk-selection kernel (cc_ppl_chunk_scores) on synthetic bf16 and
+    f32 logits of a 128256-token vocabulary, as achieved bytes/s against the HBM peak.  Two logit
+    sets larger than L2 alternate, so no call finds its input cached."""
+    import torch
+    from paper_2604_10235_b200 import binding as cc
+    chunks, t, v = 32, 64, 128256
+    out = {"shape": [chunks, t, v], "bound": "hbm", "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    tgt = torch.randint(0, v, (t,), device="cuda", dtype=torch.int32)
+    nll = torch.empty((chunks, t), device="cuda")
+    score = torch.empty((chunks,), device="cuda")
+    for name, dtype in (("bf16", torch.bfloat16), ("f32", torch.float32)):
+        gen_ = torch.Generator(device="cuda").manual_seed(7)
+        sets = [torch.randn((chunks, t, v), device="cuda", generator=gen_).to(dtype) for _ in range(2)]
+        for x in sets:
+            cc.cc_ppl_chunk_scores(ctx, x, tgt, nll, score)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 10
+        e0.record()
+        for _ in range(reps):
+            for x in sets:
+                cc.cc_ppl_chunk_scores(ctx, x, tgt, nll, score)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / (2 * reps)
+        gbs = sets[0].numel() * sets[0].element_size() / ms * 1e-6
+        out[name] = {"us": ms * 1e3, "achieved": gbs, "frac": gbs / peaks["hbm_gbs"]}
+        del sets
+    if ctx.poll() != 0:
+        raise RuntimeError("device status after the chunk-scoring measurement")
+    return out
 
 
 # DRAM bytes (read + write) of one launch pair of the score stage, from the ncu capture that

@@ -67,6 +67,7 @@ extern "C" {
 #define CC_ERR_DEVICE_FLAG  (-6)  /* device status only: a kernel met an invalid page id or index */
 
 #define CC_BF16        1
+#define CC_F32         2   /* logits of cc_ppl_chunk_scores only */
 #define CC_MODE_BF16   0   /* tensor-core scores: bf16 operands, fp32 accumulate and softmax */
 #define CC_MODE_FP32   1   /* verification mode: every product and sum in fp32 on CUDA cores */
 #define CC_POOL_NONE   0
@@ -203,6 +204,27 @@ int cc_compress_layer(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win,
 int cc_structural_score(cc_ctx* ctx, const cc_layer_desc* desc, const int32_t* idx,
                         const float* prior, float threshold, float* score, int32_t* counts,
                         void* stream);
+
+/* Chunk selection (Section 4.1 "Query-Conditioned Chunk Selection").  logits holds, for every
+ * candidate chunk i and query position t, the model's V next-token logits given prefix + C_i and
+ * the earlier query tokens: element (i, t, v) at logits[i * stride_chunk + t * stride_token + v]
+ * (device, CC_BF16 or CC_F32; strides in elements; rows that all start on 16-byte boundaries
+ * are read with vector loads, others value by value, several times slower); targets: device
+ * i32 [num_tokens], the query tokens q_t.  nll: device f32 [num_chunks][num_tokens] receives
+ * -log p(q_t | ...) = logsumexp(row) - row[q_t]; score: device f32 [num_chunks] receives their
+ * mean s_i^ppl.  A token id outside [0, V) gives NaN and CC_ERR_DEVICE_FLAG in the status word.
+ * Needs no workspace. */
+int cc_ppl_chunk_scores(cc_ctx* ctx, const void* logits, int32_t logits_dtype, int32_t num_chunks,
+                        int32_t num_tokens, int32_t vocab, int64_t stride_chunk,
+                        int64_t stride_token, const int32_t* targets, float* nll, float* score,
+                        void* stream);
+
+/* The min(k, num_chunks) chunks with the lowest score (same section: TopK of -s^ppl), written to
+ * chosen (device i32 [k]) best first; equal scores: lower index first; NaN ranks last.
+ * num_chunks <= CC_MAX_CHUNKS. */
+#define CC_MAX_CHUNKS 8192
+int cc_select_chunks(cc_ctx* ctx, const float* score, int32_t num_chunks, int32_t k,
+                     int32_t* chosen, void* stream);
 
 /* ---- host-side planning (no GPU work, no context; all pointers are HOST memory) ----------- */
 

@@ -22,6 +22,7 @@ CC_OK = 0
 CC_ERR_INVALID_ARG, CC_ERR_UNSUPPORTED, CC_ERR_WORKSPACE, CC_ERR_CUDA = -1, -2, -3, -4
 CC_ERR_TIMEOUT, CC_ERR_DEVICE_FLAG = -5, -6
 CC_BF16 = 1
+CC_F32 = 2
 CC_MODE_BF16, CC_MODE_FP32 = 0, 1
 CC_POOL_NONE, CC_POOL_MAX, CC_POOL_AVG = 0, 1, 2
 CC_MAX_SEQS = 64
@@ -29,7 +30,8 @@ CC_MAX_SEQS = 64
 EXPORTS = ("cc_create", "cc_destroy", "cc_status_string", "cc_last_error", "cc_poll_status",
            "cc_workspace_bytes", "cc_score_window", "cc_fuse_prior_pool", "cc_topk_select",
            "cc_compact_kv", "cc_compress_layer", "cc_workspace_views", "cc_topk_select_static",
-           "cc_structural_score", "cc_plan_budgets", "cc_select_spans")
+           "cc_structural_score", "cc_plan_budgets", "cc_select_spans", "cc_ppl_chunk_scores",
+           "cc_select_chunks")
 CC_STATIC_SELECT_MAX_ITEMS = 1 << 20
 
 
@@ -93,6 +95,9 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.cc_topk_select_static.argtypes = [vp, dp, vp, vp, vp, vp, vp]
     lib.cc_structural_score.argtypes = [vp, dp, vp, vp, C.c_float, vp, vp, vp]
     lib.cc_compact_kv.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.cc_ppl_chunk_scores.argtypes = [vp, vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int64,
+                                        C.c_int64, vp, vp, vp, vp]
+    lib.cc_select_chunks.argtypes = [vp, vp, C.c_int32, C.c_int32, vp, vp]
     lib.cc_plan_budgets.argtypes = [vp, vp, C.c_int32, C.POINTER(cc_budget_params), vp, vp]
     lib.cc_select_spans.argtypes = [vp, vp, vp, vp, C.c_int32, C.c_int32, C.c_int32, C.c_double,
                                     C.c_int32, vp, vp, vp]
@@ -284,6 +289,22 @@ def cc_structural_score(ctx: Context, desc: Desc, idx, prior, threshold: float, 
     ctx.check(ctx.lib.cc_structural_score(ctx.handle, C.byref(desc.c), _ptr(idx), _ptr(prior),
                                           C.c_float(threshold), _ptr(score), _ptr(counts),
                                           _stream(stream)))
+
+
+def cc_ppl_chunk_scores(ctx: Context, logits: torch.Tensor, targets: torch.Tensor,
+                        nll: torch.Tensor, score: torch.Tensor, stream=None):
+    """logits [chunks][T][V] (bf16 or f32, last dimension contiguous), targets i32 [T]."""
+    chunks, t, v = logits.shape
+    assert logits.stride(2) == 1
+    dtype = CC_F32 if logits.dtype == torch.float32 else CC_BF16
+    ctx.check(ctx.lib.cc_ppl_chunk_scores(ctx.handle, _ptr(logits), dtype, chunks, t, v,
+                                          logits.stride(0), logits.stride(1), _ptr(targets),
+                                          _ptr(nll), _ptr(score), _stream(stream)))
+
+
+def cc_select_chunks(ctx: Context, score: torch.Tensor, k: int, chosen: torch.Tensor, stream=None):
+    ctx.check(ctx.lib.cc_select_chunks(ctx.handle, _ptr(score), score.numel(), k, _ptr(chosen),
+                                       _stream(stream)))
 
 
 def _host(a: np.ndarray):

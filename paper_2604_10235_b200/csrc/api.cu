@@ -451,6 +451,44 @@ int cc_structural_score(cc_ctx* ctx, const cc_layer_desc* desc, const int32_t* i
   return CC_OK;
 }
 
+int cc_ppl_chunk_scores(cc_ctx* ctx, const void* logits, int32_t logits_dtype, int32_t num_chunks,
+                        int32_t num_tokens, int32_t vocab, int64_t stride_chunk,
+                        int64_t stride_token, const int32_t* targets, float* nll, float* score,
+                        void* stream) {
+  if (!ctx) return CC_ERR_INVALID_ARG;
+  if (logits_dtype != CC_BF16 && logits_dtype != CC_F32)
+    return fail(ctx, CC_ERR_UNSUPPORTED, "logits must be CC_BF16 or CC_F32");
+  if (num_chunks < 0 || num_tokens < 1 || vocab < 1)
+    return fail(ctx, CC_ERR_INVALID_ARG, "num_chunks >= 0, num_tokens >= 1 and vocab >= 1 are needed");
+  if (num_chunks == 0) return CC_OK;
+  if (!logits || !targets || !nll || !score) return fail(ctx, CC_ERR_INVALID_ARG, "NULL tensor pointer");
+  if ((long long)num_chunks * num_tokens > 0x7fffffffLL)
+    return fail(ctx, CC_ERR_UNSUPPORTED, "more than 2^31 rows of logits");
+  if (stride_token < vocab || stride_chunk < (int64_t)num_tokens * stride_token)
+    return fail(ctx, CC_ERR_INVALID_ARG, "strides smaller than the rows they separate");
+  if ((uintptr_t)logits % (logits_dtype == CC_F32 ? 4 : 2))
+    return fail(ctx, CC_ERR_INVALID_ARG, "logits pointer is not aligned to its element type");
+  cudaError_t e = launch_ppl_scores(make_launch(ctx, stream), logits, logits_dtype == CC_F32,
+                                    num_chunks, num_tokens, vocab, stride_chunk, stride_token,
+                                    targets, nll, score);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "perplexity score launch");
+  return CC_OK;
+}
+
+int cc_select_chunks(cc_ctx* ctx, const float* score, int32_t num_chunks, int32_t k,
+                     int32_t* chosen, void* stream) {
+  if (!ctx) return CC_ERR_INVALID_ARG;
+  if (num_chunks < 0 || k < 0) return fail(ctx, CC_ERR_INVALID_ARG, "negative count");
+  if (num_chunks > CC_MAX_CHUNKS)
+    return fail(ctx, CC_ERR_UNSUPPORTED, "more than %d chunks", CC_MAX_CHUNKS);
+  if (k > num_chunks) k = num_chunks;
+  if (k == 0) return CC_OK;
+  if (!score || !chosen) return fail(ctx, CC_ERR_INVALID_ARG, "NULL tensor pointer");
+  cudaError_t e = launch_select_chunks(make_launch(ctx, stream), score, num_chunks, k, chosen);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "chunk selection launch");
+  return CC_OK;
+}
+
 int cc_workspace_views(const cc_ctx* ctx, const cc_layer_desc* desc, void* ws, float** scores,
                        float** fused) {
   Plan p;

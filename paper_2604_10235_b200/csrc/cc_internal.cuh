@@ -151,6 +151,13 @@ cudaError_t launch_compact(const Launch& L, const BatchTable& bt, const Geometry
                            const void* k, const void* v, const int32_t* idx, void* k_out,
                            void* v_out, const int32_t* free_pages, int32_t* out_page_table);
 
+// chunk selection by query-conditioned perplexity (Section 4.1)
+cudaError_t launch_ppl_scores(const Launch& L, const void* logits, bool is_f32, int num_chunks,
+                              int num_tokens, int vocab, int64_t stride_chunk, int64_t stride_token,
+                              const int32_t* targets, float* nll, float* score);
+cudaError_t launch_select_chunks(const Launch& L, const float* score, int num_chunks, int k,
+                                 int32_t* chosen);
+
 // fraction of the critical tokens (prior >= threshold) that each head's index list retains
 cudaError_t launch_str_score(const Launch& L, const BatchTable& bt, const Geometry& g,
                              float threshold, const int32_t* idx, const float* prior,
