@@ -101,7 +101,9 @@ struct Ctx {
     if (threadIdx.x == 0) sm->xchg[b][0] = v;
     sync_all();
     unsigned t = 0;
-    for (int r = 0; r < C; ++r) t += peer(&sm->xchg[b][0], r);
+#pragma unroll
+    for (int r = 0; r < kMaxCluster; ++r)     // fixed trip count: the loads go out together
+      if (r < C) t += peer(&sm->xchg[b][0], r);
     return t;
   }
   __device__ void cluster_minmax(unsigned& lo, unsigned& hi) {
@@ -125,9 +127,12 @@ struct Ctx {
     const unsigned b = phase++ & 1u;
     if (threadIdx.x == 0) { sm->xchg[b][0] = lo; sm->xchg[b][1] = hi; }
     sync_all();
-    for (int r = 0; r < C; ++r) {
-      lo = min(lo, peer(&sm->xchg[b][0], r));
-      hi = max(hi, peer(&sm->xchg[b][1], r));
+#pragma unroll
+    for (int r = 0; r < kMaxCluster; ++r) {
+      if (r < C) {
+        lo = min(lo, peer(&sm->xchg[b][0], r));
+        hi = max(hi, peer(&sm->xchg[b][1], r));
+      }
     }
   }
   // exclusive prefix sums over the threads of the block for two counters; tot_* = block totals
@@ -165,9 +170,12 @@ struct Ctx {
     const unsigned bf = phase++ & 1u;
     if (threadIdx.x == 0) { sm->xchg[bf][0] = ta; sm->xchg[bf][1] = tb; }
     sync_all();
-    for (int r = 0; r < rank; ++r) {
-      ea += peer(&sm->xchg[bf][0], r);
-      eb += peer(&sm->xchg[bf][1], r);
+#pragma unroll
+    for (int r = 0; r < kMaxCluster - 1; ++r) {
+      if (r < rank) {
+        ea += peer(&sm->xchg[bf][0], r);
+        eb += peer(&sm->xchg[bf][1], r);
+      }
     }
   }
 };
@@ -192,12 +200,14 @@ __device__ void radix_threshold(Ctx& c, int lo, int hi, unsigned R, bool allow_e
   whole_bin = false;
   const int copy = (threadIdx.x >> 5) & (kCopies - 1);
   int shift = 32;
+#pragma unroll 1
   while (shift > 0 && range) {
     const int bits = min(kDigitBits, shift);
     const int hi_shift = shift;             // bits [31, hi_shift) are resolved
     shift -= bits;
     const unsigned b = c.phase++ & 1u;
     unsigned* h = &sm.hist[b][0][0];
+#pragma unroll 1
     for (int i = threadIdx.x; i < kCopies * kBins; i += kThreads) h[i] = 0;
     __syncthreads();
     for (int li = lo; li < hi; ++li) {
@@ -220,7 +230,9 @@ __device__ void radix_threshold(Ctx& c, int lo, int hi, unsigned R, bool allow_e
     const int bin0 = kBins - 1 - (int)threadIdx.x;
     unsigned v0 = 0;
     if (threadIdx.x < kBins)
-      for (int r = 0; r < c.C; ++r) v0 += c.peer(&sm.hist[b][0][bin0], r);
+#pragma unroll
+      for (int r = 0; r < kMaxCluster; ++r)
+        if (r < c.C) v0 += c.peer(&sm.hist[b][0][bin0], r);
     unsigned excl, d0, d1, d2;
     c.block_scan2(v0, 0u, excl, d0, d1, d2);
     if (threadIdx.x < kBins && excl < remaining && remaining <= excl + v0) {
@@ -316,6 +328,7 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
       }
       __syncthreads();
     }
+#pragma unroll 1
     for (int li = threadIdx.x; li < cta_items; li += kThreads) {
       const int i = cta_lo + li;
       float val, pr;
@@ -360,6 +373,7 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
     }
   } else {
     const float* f = P.fused_in + (int64_t)h * bt.m_tot + q.item_off;
+#pragma unroll 1
     for (int li = threadIdx.x; li < cta_items; li += kThreads) {
       keys[padded(li)] = mono_key(f[cta_lo + li]);
       flags[li] = item_prior(li) >= theta ? 1 : 0;
@@ -369,6 +383,7 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
 
   // ---- stage 0: protected weight
   unsigned wf = 0;
+#pragma unroll 1
   for (int li = lo; li < hi; ++li) if (flags[li]) wf += item_len(li);
   unsigned forced_tokens = c.cluster_sum(wf);
 
@@ -385,11 +400,13 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
                       return true;
                     }, t1, above1, whole);
     unsigned tie_w = 0;
+#pragma unroll 1
     for (int li = lo; li < hi; ++li)
       if (flags[li] && mono_key(item_prior(li)) == t1) tie_w += item_len(li);
     unsigned tie_before, dummy;
     c.cluster_scan2(tie_w, 0u, tie_before, dummy);
     unsigned kept = 0;
+#pragma unroll 1
     for (int li = lo; li < hi; ++li) {
       if (!flags[li]) continue;
       const unsigned key = mono_key(item_prior(li));
@@ -426,6 +443,7 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
 
   // ---- stage 3: ordered emission
   unsigned def_w = 0, tie_w = 0;
+#pragma unroll 1
   for (int li = lo; li < hi; ++li) {
     const unsigned len = item_len(li);
     if (flags[li]) {
@@ -440,6 +458,7 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
   // last read of a peer's shared memory is done: announce it now, wait for the peers at the
   // very end, and write the indices in between
   if (c.C > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+#pragma unroll 1
   for (int li = lo; li < hi; ++li) {
     const unsigned len = item_len(li);
     unsigned take = 0;
