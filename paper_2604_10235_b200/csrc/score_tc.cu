@@ -323,7 +323,7 @@ struct Pipe {
 };
 
 // Bounded wait; false (and the abort flag set) when the bound is hit or another role gave up.
-__device__ __forceinline__ bool wait_bar(const Pipe& p, uint64_t* bar, uint32_t parity, int where) {
+__device__ __noinline__ bool wait_bar(const Pipe& p, uint64_t* bar, uint32_t parity, int where) {
   const uint32_t b = smem_u32(bar);
   for (uint32_t i = 0; i < 4000000u; ++i) {
     if (mbar_try_wait(b, parity)) return true;
@@ -850,6 +850,7 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
   // ---------------------------------------------------------------- teardown
   if (misc->abort_flag) {
     // give copies still in flight time to land before shared memory is released
+#pragma unroll 1
     for (int i = 0; i < 2000; ++i) __nanosleep(1000);
   }
   tc_fence_before();
