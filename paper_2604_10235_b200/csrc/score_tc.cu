@@ -414,7 +414,12 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = misc->tmem_base;
-  pdl_wait();
+  // Pass 1 reads Q and K, which the launch before it in the stream may have produced: every
+  // thread waits for that launch.  The launch before pass 2 is pass 1, which only produces the
+  // row statistics: the TMA and MMA roles of pass 2 start at once (their first K tiles and
+  // products overlap the tail of pass 1) and only the epilogue warps, which read the statistics
+  // and write the scores, wait.
+  if (PASS == 1) pdl_wait();
 
   if (warp == 0) {
     // ================================================================ TMA producer
@@ -690,6 +695,7 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
     const uint32_t full_bar = smem_u32(&misc->bar.acc_full[set]);
     const uint32_t empty_bar = smem_u32(&misc->bar.acc_empty[set]);
     const uint32_t acc_addr = lane_addr + (uint32_t)set * kBufCols;
+    if (PASS == 2) pdl_wait();
     for (;;) {
       if (t >= prob_end) {
         bool done = false;
