@@ -409,17 +409,21 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
     tmem_alloc(smem_u32(&misc->tmem_base), kTmemCols);
     tmem_relinquish();
   }
-  pdl_launch_dependents();
+  if (PASS == 2) pdl_launch_dependents();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = misc->tmem_base;
   // Pass 1 reads Q and K, which the launch before it in the stream may have produced: every
-  // thread waits for that launch.  The launch before pass 2 is pass 1, which only produces the
-  // row statistics: the TMA and MMA roles of pass 2 start at once (their first K tiles and
-  // products overlap the tail of pass 1) and only the epilogue warps, which read the statistics
-  // and write the scores, wait.
-  if (PASS == 1) pdl_wait();
+  // thread waits for that launch, and only then lets pass 2 be scheduled, so that whatever runs
+  // after pass 1 has begun finds the caller's inputs complete.  The launch before pass 2 is
+  // pass 1, which only produces the row statistics: the TMA and MMA roles of pass 2 start at
+  // once (their first K tiles and products overlap the tail of pass 1) and only the epilogue
+  // warps, which read the statistics and write the scores, wait.
+  if (PASS == 1) {
+    pdl_wait();
+    pdl_launch_dependents();
+  }
 
   if (warp == 0) {
     // ================================================================ TMA producer

@@ -267,7 +267,10 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
   c.phase = 0;
 
   pdl_launch_dependents();
-  pdl_wait();
+  // FUSED runs right after the second score pass, which starts only once the caller's inputs
+  // are complete: the token-level path reads the prior before it waits for the scores
+  const bool early_prior = FUSED && bt.chunk == 1;
+  if (!early_prior) pdl_wait();
 
   const int h = blockIdx.y, s = blockIdx.z;
   const SeqInfo& q = bt.seq[s];
@@ -311,20 +314,27 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
       // the key slots; four loads of each are issued before the first store, so the slice
       // costs a couple of round trips to L2 instead of one per item
       const int span = cta_items + 2 * half;
+#pragma unroll 1
+      for (int t0 = threadIdx.x; t0 < cta_items; t0 += 4 * kThreads) {
+        float b[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) b[k] = t0 + k * kThreads < cta_items ? p[cta_lo + t0 + k * kThreads] : 0.0f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (t0 + k * kThreads < cta_items) keys[padded(t0 + k * kThreads)] = __float_as_uint(b[k]);
+      }
+      pdl_wait();                                   // the scores are complete from here on
+#pragma unroll 1
       for (int t0 = threadIdx.x; t0 < span; t0 += 4 * kThreads) {
-        float a[4], b[4];
+        float a[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const int t = t0 + k * kThreads, j = cta_lo - half + t;
           a[k] = (t < span && j >= 0 && j < q.n) ? u[j] : 0.0f;
-          b[k] = t < cta_items ? p[cta_lo + t] : 0.0f;
         }
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const int t = t0 + k * kThreads;
-          if (t < span) us[t] = a[k];
-          if (t < cta_items) keys[padded(t)] = __float_as_uint(b[k]);
-        }
+        for (int k = 0; k < 4; ++k)
+          if (t0 + k * kThreads < span) us[t0 + k * kThreads] = a[k];
       }
       __syncthreads();
     }
