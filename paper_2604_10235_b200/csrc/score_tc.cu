@@ -388,6 +388,11 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t_begin = span_begin(blockIdx.x, P), t_end = span_begin(blockIdx.x + 1, P);
 
+  if (threadIdx.x == 32) {
+    // fetch the two TMA descriptors (kernel parameters) while the barriers are being set up
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&q_map)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&k_map)) : "memory");
+  }
   if (threadIdx.x == 0) {
     for (int i = 0; i < kMaxStages; ++i) {
       mbar_init(smem_u32(&misc->bar.full[i]), 1);
