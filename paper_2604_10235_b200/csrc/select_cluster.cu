@@ -254,7 +254,9 @@ __device__ void radix_threshold(Ctx& c, int lo, int hi, unsigned R, bool allow_e
   if (whole_bin) w_above = R;
 }
 
-template <bool FUSED>
+// CHUNKED instantiations rank fixed chunks of bt.chunk tokens; the others are compiled for
+// token-level items only (bt.chunk == 1), which keeps their code short.
+template <bool FUSED, bool CHUNKED>
 __global__ void __launch_bounds__(kThreads, 1)
 select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ ClusterParams P) {
   extern __shared__ __align__(16) uint8_t dyn[];
@@ -269,12 +271,12 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
   pdl_launch_dependents();
   // FUSED runs right after the second score pass, which starts only once the caller's inputs
   // are complete: the token-level path reads the prior before it waits for the scores
-  const bool early_prior = FUSED && bt.chunk == 1;
+  const bool early_prior = FUSED && !CHUNKED;
   if (!early_prior) pdl_wait();
 
   const int h = blockIdx.y, s = blockIdx.z;
   const SeqInfo& q = bt.seq[s];
-  const int m = q.n_items, cs = bt.chunk;
+  const int m = q.n_items, cs = CHUNKED ? bt.chunk : 1;
   const int per = (m + c.C * kThreads - 1) / (c.C * kThreads);       // items per thread
   const int cta_lo = min(m, c.rank * kThreads * per);
   const int cta_hi = min(m, cta_lo + kThreads * per);
@@ -541,7 +543,9 @@ cudaError_t launch_select_cluster(const Launch& L, const BatchTable& bt, const G
   P.count = count;
   const int per = bt.max_items > 0 ? (bt.max_items + cluster * kThreads - 1) / (cluster * kThreads) : 1;
   const size_t smem = cluster_smem_bytes(per, fused_input, P.pool_size);
-  auto kern = fused_input ? select_cluster_kernel<true> : select_cluster_kernel<false>;
+  const bool chunked = bt.chunk > 1;
+  auto kern = fused_input ? (chunked ? select_cluster_kernel<true, true> : select_cluster_kernel<true, false>)
+                          : (chunked ? select_cluster_kernel<false, true> : select_cluster_kernel<false, false>);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   return launch_pdl(kern, dim3(cluster, g.hkv, bt.num_seqs), dim3(kThreads), smem, L.stream, cluster, bt, P);
