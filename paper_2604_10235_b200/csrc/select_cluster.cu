@@ -162,6 +162,25 @@ struct Ctx {
     ea = __shfl_sync(0xffffffffu, xa - wa, warp) + ia - a;
     eb = __shfl_sync(0xffffffffu, xb - wb, warp) + ib - b;
   }
+  // exclusive prefix of one counter over all threads of the cluster, and its cluster total
+  __device__ void cluster_scan_total(unsigned a, unsigned& ea, unsigned& total) {
+    unsigned eb, ta, tb;
+    block_scan2(a, 0u, ea, eb, ta, tb);
+    total = ta;
+    if (C == 1) return;
+    const unsigned bf = phase++ & 1u;
+    if (threadIdx.x == 0) sm->xchg[bf][0] = ta;
+    sync_all();
+    total = 0;
+#pragma unroll
+    for (int r = 0; r < kMaxCluster; ++r) {
+      if (r < C) {
+        const unsigned v = peer(&sm->xchg[bf][0], r);
+        total += v;
+        if (r < rank) ea += v;
+      }
+    }
+  }
   // the same over all threads of the cluster (CTA rank major)
   __device__ void cluster_scan2(unsigned a, unsigned b, unsigned& ea, unsigned& eb) {
     unsigned ta, tb;
@@ -397,10 +416,15 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
   unsigned wf = 0;
 #pragma unroll 1
   for (int li = lo; li < hi; ++li) if (flags[li]) wf += item_len(li);
-  unsigned forced_tokens = c.cluster_sum(wf);
+  // the prefix comes with the sum: when the protected items alone fill the budget it is all
+  // the emission needs, and the scan of stage 3 is skipped
+  unsigned forced_before, forced_tokens;
+  c.cluster_scan_total(wf, forced_before, forced_tokens);
+  bool flags_as_counted = true;
 
   // ---- stage 1: cap on protected items (longest prefix by (prior desc, index asc) within B_span)
   if (q.span_cap >= 0 && forced_tokens > (unsigned)q.span_cap) {
+    flags_as_counted = false;
     const unsigned cap = (unsigned)q.span_cap;
     unsigned t1, above1;
     bool whole;
@@ -454,7 +478,9 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
   }
 
   // ---- stage 3: ordered emission
+  const bool reuse_prefix = ties_are_forced && flags_as_counted;
   unsigned def_w = 0, tie_w = 0;
+  if (!reuse_prefix) {
 #pragma unroll 1
   for (int li = lo; li < hi; ++li) {
     const unsigned len = item_len(li);
@@ -465,8 +491,14 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
       if (key > t || (whole_bin && key == t)) def_w += len; else if (key == t) tie_w += len;
     }
   }
+  }
   unsigned def_before, tie_before;
-  c.cluster_scan2(def_w, tie_w, def_before, tie_before);
+  if (reuse_prefix) {
+    def_before = 0;
+    tie_before = forced_before;
+  } else {
+    c.cluster_scan2(def_w, tie_w, def_before, tie_before);
+  }
   // last read of a peer's shared memory is done: announce it now, wait for the peers at the
   // very end, and write the indices in between
   if (c.C > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
