@@ -37,7 +37,7 @@ constexpr int kCtaItems = 16384;          // items one CTA keeps in shared memor
 
 struct Shared {
   unsigned hist[2][kCopies][kBins];
-  unsigned xchg[2][4];
+  unsigned xchg[2][kMaxCluster][4];   // [buffer copy][source CTA][word]: written by the peers
   unsigned warp_a[kWarps];
   unsigned warp_b[kWarps];
   unsigned bcast[4];
@@ -84,6 +84,23 @@ struct Ctx {
     return *cg::this_cluster().map_shared_rank(const_cast<unsigned*>(p), r);
   }
 
+  // Exchange of up to three words per CTA: threads 0..C-1 each store this CTA's words into one
+  // peer's shared memory (remote stores need no round trip), the cluster barrier publishes them,
+  // and every thread then reads all CTAs' words locally.  Two buffer copies: a CTA writes copy
+  // k & 1 for exchange k only after the barrier of exchange k - 1, which every peer reaches
+  // after it has read exchange k - 2.
+  __device__ unsigned publish(unsigned w0, unsigned w1, unsigned w2) {
+    const unsigned bf = phase++ & 1u;
+    if ((int)threadIdx.x < C) {
+      unsigned* dst = cg::this_cluster().map_shared_rank(&sm->xchg[bf][rank][0], (int)threadIdx.x);
+      dst[0] = w0;
+      dst[1] = w1;
+      dst[2] = w2;
+    }
+    sync_all();
+    return bf;
+  }
+
   // sum over the block; every thread gets the result
   __device__ unsigned block_sum(unsigned v) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -97,13 +114,11 @@ struct Ctx {
   __device__ unsigned cluster_sum(unsigned v) {
     v = block_sum(v);
     if (C == 1) return v;
-    const unsigned b = phase++ & 1u;
-    if (threadIdx.x == 0) sm->xchg[b][0] = v;
-    sync_all();
+    const unsigned b = publish(v, 0u, 0u);
     unsigned t = 0;
 #pragma unroll
-    for (int r = 0; r < kMaxCluster; ++r)     // fixed trip count: the loads go out together
-      if (r < C) t += peer(&sm->xchg[b][0], r);
+    for (int r = 0; r < kMaxCluster; ++r)
+      if (r < C) t += sm->xchg[b][r][0];
     return t;
   }
   __device__ void cluster_minmax(unsigned& lo, unsigned& hi) {
@@ -124,14 +139,12 @@ struct Ctx {
       hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, o));
     }
     if (C == 1) return;
-    const unsigned b = phase++ & 1u;
-    if (threadIdx.x == 0) { sm->xchg[b][0] = lo; sm->xchg[b][1] = hi; }
-    sync_all();
+    const unsigned b = publish(lo, hi, 0u);
 #pragma unroll
     for (int r = 0; r < kMaxCluster; ++r) {
       if (r < C) {
-        lo = min(lo, peer(&sm->xchg[b][0], r));
-        hi = max(hi, peer(&sm->xchg[b][1], r));
+        lo = min(lo, sm->xchg[b][r][0]);
+        hi = max(hi, sm->xchg[b][r][1]);
       }
     }
   }
@@ -168,14 +181,12 @@ struct Ctx {
     block_scan2(a, 0u, ea, eb, ta, tb);
     total = ta;
     if (C == 1) return;
-    const unsigned bf = phase++ & 1u;
-    if (threadIdx.x == 0) sm->xchg[bf][0] = ta;
-    sync_all();
+    const unsigned bf = publish(ta, 0u, 0u);
     total = 0;
 #pragma unroll
     for (int r = 0; r < kMaxCluster; ++r) {
       if (r < C) {
-        const unsigned v = peer(&sm->xchg[bf][0], r);
+        const unsigned v = sm->xchg[bf][r][0];
         total += v;
         if (r < rank) ea += v;
       }
@@ -186,14 +197,12 @@ struct Ctx {
     unsigned ta, tb;
     block_scan2(a, b, ea, eb, ta, tb);
     if (C == 1) return;
-    const unsigned bf = phase++ & 1u;
-    if (threadIdx.x == 0) { sm->xchg[bf][0] = ta; sm->xchg[bf][1] = tb; }
-    sync_all();
+    const unsigned bf = publish(ta, tb, 0u);
 #pragma unroll
     for (int r = 0; r < kMaxCluster - 1; ++r) {
       if (r < rank) {
-        ea += peer(&sm->xchg[bf][0], r);
-        eb += peer(&sm->xchg[bf][1], r);
+        ea += sm->xchg[bf][r][0];
+        eb += sm->xchg[bf][r][1];
       }
     }
   }
