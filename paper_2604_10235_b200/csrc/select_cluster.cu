@@ -176,12 +176,30 @@ struct Ctx {
     eb = __shfl_sync(0xffffffffu, xb - wb, warp) + ib - b;
   }
   // exclusive prefix of one counter over all threads of the cluster, and its cluster total
-  __device__ void cluster_scan_total(unsigned a, unsigned& ea, unsigned& total) {
+  // and, in the same exchange, the cluster-wide minimum of lo and maximum of hi (carried through
+  // the block scan as its second counter's inputs would not do: they are reduced separately)
+  __device__ void cluster_scan_total(unsigned a, unsigned& ea, unsigned& total, unsigned& lo,
+                                     unsigned& hi) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    __shared__ unsigned w_lo[kWarps], w_hi[kWarps];
+    if (lane == 0) { w_lo[warp] = lo; w_hi[warp] = hi; }
     unsigned eb, ta, tb;
-    block_scan2(a, 0u, ea, eb, ta, tb);
+    block_scan2(a, 0u, ea, eb, ta, tb);      // its barriers also publish w_lo / w_hi
+    lo = w_lo[lane];
+    hi = w_hi[lane];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
     total = ta;
     if (C == 1) return;
-    const unsigned bf = publish(ta, 0u, 0u);
+    const unsigned bf = publish(ta, lo, hi);
     total = 0;
 #pragma unroll
     for (int r = 0; r < kMaxCluster; ++r) {
@@ -189,6 +207,8 @@ struct Ctx {
         const unsigned v = sm->xchg[bf][r][0];
         total += v;
         if (r < rank) ea += v;
+        lo = min(lo, sm->xchg[bf][r][1]);
+        hi = max(hi, sm->xchg[bf][r][2]);
       }
     }
   }
@@ -214,14 +234,17 @@ struct Ctx {
 // with key >= T is taken and nothing is tied.  w_above = weight strictly above the ties.
 template <class Get>
 __device__ void radix_threshold(Ctx& c, int lo, int hi, unsigned R, bool allow_early, Get get,
-                                unsigned& T, unsigned& w_above, bool& whole_bin) {
+                                unsigned& T, unsigned& w_above, bool& whole_bin,
+                                bool range_known = false, unsigned kmin = 0xffffffffu,
+                                unsigned kmax = 0u) {
   Shared& sm = *c.sm;
-  unsigned kmin = 0xffffffffu, kmax = 0u;
-  for (int li = lo; li < hi; ++li) {
-    unsigned key, len;
-    if (get(li, key, len)) { kmin = min(kmin, key); kmax = max(kmax, key); }
+  if (!range_known) {
+    for (int li = lo; li < hi; ++li) {
+      unsigned key, len;
+      if (get(li, key, len)) { kmin = min(kmin, key); kmax = max(kmax, key); }
+    }
+    c.cluster_minmax(kmin, kmax);
   }
-  c.cluster_minmax(kmin, kmax);
   const unsigned range = kmax - kmin;
   const int sh = range ? __clz(range) : 0;
   unsigned prefix = 0, remaining = R;
@@ -422,13 +445,21 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
   __syncthreads();
 
   // ---- stage 0: protected weight
-  unsigned wf = 0;
+  unsigned wf = 0, free_min = 0xffffffffu, free_max = 0u;   // key range of the unprotected items
 #pragma unroll 1
-  for (int li = lo; li < hi; ++li) if (flags[li]) wf += item_len(li);
-  // the prefix comes with the sum: when the protected items alone fill the budget it is all
-  // the emission needs, and the scan of stage 3 is skipped
+  for (int li = lo; li < hi; ++li) {
+    if (flags[li]) {
+      wf += item_len(li);
+    } else {
+      const unsigned key = keys[padded(li)];
+      free_min = min(free_min, key);
+      free_max = max(free_max, key);
+    }
+  }
+  // one exchange yields the sum, its prefix (all the emission needs when the protected items
+  // alone fill the budget: the scan of stage 3 is skipped) and the key range of stage 2
   unsigned forced_before, forced_tokens;
-  c.cluster_scan_total(wf, forced_before, forced_tokens);
+  c.cluster_scan_total(wf, forced_before, forced_tokens, free_min, free_max);
   bool flags_as_counted = true;
 
   // ---- stage 1: cap on protected items (longest prefix by (prior desc, index asc) within B_span)
@@ -482,7 +513,7 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
                       key = keys[padded(li)];
                       len = item_len(li);
                       return true;
-                    }, t, above, whole_bin);
+                    }, t, above, whole_bin, flags_as_counted, free_min, free_max);
     tie_budget = keep - forced_tokens - above;
   }
 
