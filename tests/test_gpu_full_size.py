@@ -27,3 +27,13 @@ def test_ragged_paged_full_size():
     output into fresh pages."""
     wl = gen.workloads()["ragged_paged"]
     check_layer(wl, gen.make_layer(wl), cc.CC_MODE_BF16, 2e-3)
+
+
+@pytest.mark.parametrize("density", ["5", "15", "30"])
+@pytest.mark.parametrize("budget", [1024, 4096, 8192])
+def test_qwen_shape_budget_and_prior_density_sweep(budget, density):
+    """65536 tokens, 28 / 4 heads: budgets below and above the number of protected tokens (5 %
+    of the tokens = 3277 protected: the attention scores fill the rest for B = 4096 and 8192;
+    15 % and 30 % exceed every budget, so the first B protected tokens are kept)."""
+    wl = gen.qwen_variant(gen.workloads()["qwen25_coder_7b"], budget, density)
+    check_layer(wl, gen.make_layer(wl, layer=2), cc.CC_MODE_BF16, 2e-3)
