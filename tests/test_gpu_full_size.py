@@ -37,3 +37,32 @@ def test_qwen_shape_budget_and_prior_density_sweep(budget, density):
     15 % and 30 % exceed every budget, so the first B protected tokens are kept)."""
     wl = gen.qwen_variant(gen.workloads()["qwen25_coder_7b"], budget, density)
     check_layer(wl, gen.make_layer(wl, layer=2), cc.CC_MODE_BF16, 2e-3)
+
+
+def test_llama_shape_weighted_prior_mode_full_size():
+    """The prior as a weighted term of the score (attention weight 0.06, Appendix "Structural prior
+    configuration") with protection off, at the Llama-shaped size."""
+    from dataclasses import replace
+    wl = gen.workloads()["llama3_8b"]
+    wl = replace(wl, alpha=0.06 / (wl.window * wl.group), beta=1.0, force_threshold=float("inf"))
+    check_layer(wl, gen.make_layer(wl, layer=3), cc.CC_MODE_BF16, 2e-3)
+
+
+@pytest.mark.parametrize("ratio,smin", [(0.5, 16), (1.0, 0)])
+def test_llama_shape_selection_with_span_cap_full_size(ratio, smin):
+    """Selection stage alone, bit for bit, at n = 32768 with the benchmark prior (2178 protected
+    tokens against B = 2048): with rho = 0.5 the protected set is cut to B_span = 1024 and the
+    attention scores fill the rest."""
+    import numpy as np
+    from oracle import codecomp_oracle as orc
+    from test_gpu_stages import run_select
+    wl = gen.workloads()["llama3_8b"]
+    x = gen.make_layer(wl, layer=4, with_v=False)
+    rng = np.random.Generator(np.random.PCG64(8))
+    u = (np.abs(rng.standard_normal((wl.n_heads_kv, wl.n))) * 1e-3).astype(np.float32)
+    fused = orc.pool_scores(u, orc.POOL_MAX, 7, dtype=np.float32)
+    idx, count = run_select(fused, x.prior, wl.n, wl.budget, wl.force_threshold, ratio, smin)
+    for h in range(wl.n_heads_kv):
+        ref = orc.select_tokens(fused[h], x.prior, wl.n, wl.budget, wl.force_threshold, ratio, smin)
+        assert count[h] == len(ref) == wl.budget
+        np.testing.assert_array_equal(idx[h, :len(ref)], ref)
