@@ -401,7 +401,7 @@ def chunk_scoring_bandwidth(ctx, peaks):
 
 
 # DRAM bytes (read + write) of one launch pair of the score stage, from the ncu capture that
-# profiles/score_tc_kernel_llama3_8b.md summarises (llama3_8b: 67.67 + 0.81 MB for pass 1,
+# is summarised under profiles/ (llama3_8b: 67.67 + 0.81 MB for pass 1,
 # 68.00 + 1.44 MB for pass 2).  The counters were taken on the kernel as it stands in this tree;
 # other workloads have no capture and report null.
 SCORE_TRAFFIC_BYTES = {"llama3_8b": 137.93e6}
