@@ -165,9 +165,9 @@ int cc_topk_select(cc_ctx* ctx, const cc_layer_desc* desc, const float* fused,
  * inside the library's device image: CC_STATIC_SELECT_MAX_ITEMS bytes on every GPU that loads
  * the library, held until the process exits.  Calls with n_heads_kv * (total items of the
  * batch) above that limit fail with CC_ERR_UNSUPPORTED and enqueue nothing.  The call
- * allocates and frees nothing.  Its first use on a device looks up the array's device address
- * (the context's device must be the current device); make that first call outside any stream
- * capture.  All calls, from every context and stream, share the one array: two calls whose
+ * allocates and frees nothing.  The context's device must be the current device on every call
+ * (CC_ERR_INVALID_ARG otherwise).  Its first use on a device looks up the array's device
+ * address; make that first call outside any stream capture.  All calls, from every context and stream, share the one array: two calls whose
  * kernels may run at the same time on the GPU race, so keep them ordered (one stream, or
  * events).  Nothing needs clearing between calls: every flag is written before it is read.
  * Inputs and outputs are exactly those of cc_topk_select. */

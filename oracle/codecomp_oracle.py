@@ -181,23 +181,13 @@ def span_budget(budget: int, span_ratio: float, span_min: int) -> int:
     return int(min(budget, max(span_min, math.floor(span_ratio * budget + 1e-9))))
 
 
-def select_items(fused: np.ndarray, prior: np.ndarray, lens: np.ndarray, budget: int,
-                 force_threshold: float, span_ratio: float = 0.0, span_min: int = 0
-                 ) -> np.ndarray:
-    """How many leading tokens of each item (token or chunk) are retained.
-
-    Items are ranked by: protected first (among themselves by position), then larger
-    fused score, then smaller index.
-    Items are taken in rank order until ``min(budget, total tokens)`` tokens are kept;
-    the item that crosses the budget keeps only its first tokens.  Protected items are
-    those with prior >= force_threshold; with span_ratio > 0 they are limited to the
-    longest prefix, ranked by (prior descending, index ascending), whose token count
-    stays within B^span.
-    """
-    m = len(fused)
+def protected_items(prior: np.ndarray, lens: np.ndarray, budget: int, force_threshold: float,
+                    span_ratio: float = 0.0, span_min: int = 0) -> np.ndarray:
+    """Mask of the protected items (Section 4.4, "Token-level protection" and "Span selection
+    under budget"): prior >= force_threshold; with span_ratio > 0 only the longest prefix of
+    them, ranked by (prior descending, index ascending), whose token count stays within B^span."""
+    m = len(prior)
     lens = np.asarray(lens, dtype=np.int64)
-    total = int(lens.sum())
-    b_eff = max(0, min(int(budget), total))
     idx = np.arange(m)
     # the prior is an fp32 input, so the threshold test is an fp32 comparison
     forced = np.asarray(prior).astype(np.float32) >= np.float32(force_threshold)
@@ -208,6 +198,26 @@ def select_items(fused: np.ndarray, prior: np.ndarray, lens: np.ndarray, budget:
         cum = np.cumsum(lens[order])
         forced = np.zeros(m, dtype=bool)
         forced[order[cum <= cap]] = True
+    return forced
+
+
+def select_items(fused: np.ndarray, prior: np.ndarray, lens: np.ndarray, budget: int,
+                 force_threshold: float, span_ratio: float = 0.0, span_min: int = 0
+                 ) -> np.ndarray:
+    """How many leading tokens of each item (token or chunk) are retained.
+
+    Items are ranked by: protected first (among themselves by position), then larger
+    fused score, then smaller index.
+    Items are taken in rank order until ``min(budget, total tokens)`` tokens are kept;
+    the item that crosses the budget keeps only its first tokens.  Protected items are
+    those of ``protected_items``.
+    """
+    m = len(fused)
+    lens = np.asarray(lens, dtype=np.int64)
+    total = int(lens.sum())
+    b_eff = max(0, min(int(budget), total))
+    idx = np.arange(m)
+    forced = protected_items(prior, lens, budget, force_threshold, span_ratio, span_min)
     f = np.asarray(fused, dtype=np.float64) + 0.0          # -0.0 ranks equal to +0.0
     f = np.where(forced, np.inf, f)                        # protected items rank by position only
     order = np.lexsort((idx, -f, ~forced))                 # last key is the primary one

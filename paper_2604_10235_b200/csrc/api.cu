@@ -153,6 +153,7 @@ int build_plan(cc_ctx* ctx, const cc_layer_desc* d, Plan* p) {
   g.page_table = d->page_table;
   g.page_table_stride = d->page_table_stride;
   g.out_page_table_stride = d->out_page_table_stride;
+  g.pool_pages = d->pool_pages;
 
   size_t off = 0;
   p->off_scores = off;    off += align256((size_t)g.hkv * bt.n_tot * sizeof(float));

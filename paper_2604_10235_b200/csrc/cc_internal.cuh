@@ -47,7 +47,7 @@ struct Geometry {
   const int32_t* page_table;
   int page_table_stride, out_page_table_stride;
   int causal;      // window rows are the last w tokens of the sequence: row t sees keys <= n - w + t
-  int pad_;
+  int pool_pages;  // pages in the K/V pool (paged layout): page ids must lie in [0, pool_pages)
 };
 
 // Device status word: [0] = first error code, [1] = detail (where it happened).
@@ -61,14 +61,13 @@ __device__ __forceinline__ void report_error(DeviceStatus* st, int code, int det
   if (atomicCAS(&st->code, 0, code) == 0) st->detail = detail;
 }
 
-// Pool row of token j of a sequence (paged or contiguous).  Returns -1 for a bad page id.
-__device__ __forceinline__ int64_t token_row(const BatchTable& bt, const Geometry& g, int s, int j,
-                                             int64_t pool_rows) {
+// Pool row of token j of a sequence (paged or contiguous).  Returns -1 for a page id outside
+// [0, pool_pages): the caller skips the access and records CC_ERR_DEVICE_FLAG.
+__device__ __forceinline__ int64_t token_row(const BatchTable& bt, const Geometry& g, int s, int j) {
   if (bt.page_size == 0) return (int64_t)bt.seq[s].tok_off + j;
-  int page = g.page_table[(int64_t)s * g.page_table_stride + j / bt.page_size];
-  int64_t row = (int64_t)page * bt.page_size + j % bt.page_size;
-  if (page < 0 || (pool_rows > 0 && row >= pool_rows)) return -1;
-  return row;
+  const int page = g.page_table[(int64_t)s * g.page_table_stride + j / bt.page_size];
+  if (page < 0 || page >= g.pool_pages) return -1;
+  return (int64_t)page * bt.page_size + j % bt.page_size;
 }
 
 struct Launch {

@@ -39,9 +39,14 @@ compact_kernel(const __grid_constant__ BatchTable bt, const Geometry g,
   // the block with index 0 of each sequence also publishes the sequence's new page table
   if (ps > 0 && blockIdx.x == 0) {
     const int used = (q.keep + ps - 1) / ps;
-    for (int i = threadIdx.x; i < g.out_page_table_stride; i += kThreads)
-      out_page_table[(int64_t)s * g.out_page_table_stride + i] =
-          i < used ? free_pages[q.out_page_off + i] : -1;
+    for (int i = threadIdx.x; i < g.out_page_table_stride; i += kThreads) {
+      int page = i < used ? free_pages[q.out_page_off + i] : -1;
+      if (i < used && (page < 0 || page >= g.pool_pages)) {     // never published, never written
+        report_error(status, CC_ERR_DEVICE_FLAG, 503);
+        page = -1;
+      }
+      out_page_table[(int64_t)s * g.out_page_table_stride + i] = page;
+    }
   }
 
   const int64_t pairs = (int64_t)q.keep * g.hkv;
@@ -54,7 +59,7 @@ compact_kernel(const __grid_constant__ BatchTable bt, const Geometry g,
       if (lane == 0) report_error(status, CC_ERR_DEVICE_FLAG, 500);
       continue;
     }
-    const int64_t src_row = token_row(bt, g, s, tok, 0);
+    const int64_t src_row = token_row(bt, g, s, tok);
     if (src_row < 0) {
       if (lane == 0) report_error(status, CC_ERR_DEVICE_FLAG, 501);
       continue;
@@ -64,7 +69,7 @@ compact_kernel(const __grid_constant__ BatchTable bt, const Geometry g,
       dst = ((int64_t)q.idx_off + slot) * g.out_stride_tok + (int64_t)h * g.out_stride_head;
     } else {
       const int page = free_pages[q.out_page_off + slot / ps];
-      if (page < 0) {
+      if (page < 0 || page >= g.pool_pages) {
         if (lane == 0) report_error(status, CC_ERR_DEVICE_FLAG, 502);
         continue;
       }

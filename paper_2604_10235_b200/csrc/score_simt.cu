@@ -92,7 +92,7 @@ score_simt_kernel(const __grid_constant__ BatchTable bt, const Geometry g, const
       const int j = e / (kHeadDim / 8), part = e % (kHeadDim / 8);
       uint4 v = make_uint4(0, 0, 0, 0);
       if (j < valid) {
-        const int64_t row = token_row(bt, g, s, base + j, 0);
+        const int64_t row = token_row(bt, g, s, base + j);
         if (row < 0) {
           report_error(status, CC_ERR_DEVICE_FLAG, 100);
         } else {

@@ -323,12 +323,26 @@ struct Pipe {
 };
 
 // Bounded wait; false (and the abort flag set) when the bound is hit or another role gave up.
+// A healthy wait lasts microseconds; the bound is 50 ms of wall-clock time (the global timer is
+// read only after the first probes have failed, and then once every eight probes).
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
 __device__ __noinline__ bool wait_bar(const Pipe& p, uint64_t* bar, uint32_t parity, int where) {
   const uint32_t b = smem_u32(bar);
-  for (uint32_t i = 0; i < 4000000u; ++i) {
+  for (int i = 0; i < 64; ++i)
     if (mbar_try_wait(b, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 8; ++i) {
+      if (mbar_try_wait(b, parity)) return true;
+      __nanosleep(200);
+    }
     if (p.misc->abort_flag) return false;
-    if (i > 64) __nanosleep(200);
+    if (global_ns() - t0 > 50ull * 1000 * 1000) break;
   }
   p.misc->abort_flag = 1;
   report_error(p.status, CC_ERR_TIMEOUT, where);

@@ -287,14 +287,16 @@ cudaError_t launch_select_static(const Launch& L, const BatchTable& bt, const Ge
                                  int32_t* idx, int32_t* count, int device) {
   // In host code the array's name is only a handle; its device address is looked up once per
   // device (with that device current) and cached.
+  // The launch goes to the current device, so that has to be the context's device on every
+  // call, not only on the one that resolves the address.
   static uint8_t* cached[64] = {nullptr};
   if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
+  int cur = -1;
+  cudaError_t e = cudaGetDevice(&cur);
+  if (e != cudaSuccess) return e;
+  if (cur != device) return cudaErrorInvalidDevice;
   uint8_t* ptr = cached[device];
   if (ptr == nullptr) {
-    int cur = -1;
-    cudaError_t e = cudaGetDevice(&cur);
-    if (e != cudaSuccess) return e;
-    if (cur != device) return cudaErrorInvalidDevice;
     e = cudaGetSymbolAddress((void**)&ptr, g_static_select_flags);
     if (e != cudaSuccess) return e;
     if (ptr == nullptr) return cudaErrorInvalidSymbol;

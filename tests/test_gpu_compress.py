@@ -66,8 +66,10 @@ def check_layer(wl, x, mode, tol):
                                     wl.span_ratio, wl.span_min, chunk, causal=wl.causal)
         assert_scores_close(got["scores"][:, lo:lo + n], ref["scores"], rows, n, tol)
         m = len(ref["item_prior"])
-        forced_items = ref["item_prior"].astype(np.float32) >= np.float32(wl.force_threshold)
-        assert wl.span_ratio == 0.0          # the band check below assumes uncapped protection
+        # the protected set (capped to the span budget when a span ratio is set) depends on the
+        # prior alone, so it is taken from the oracle; what the scores decide is checked below
+        forced_items = orc.protected_items(ref["item_prior"], orc.chunk_lengths(n, chunk), b,
+                                           wl.force_threshold, wl.span_ratio, wl.span_min)
         # how far a fused value may move when every score in its pooling window (or chunk)
         # moves by its tolerance: alpha * (sum or max of the per-score bounds)
         tol_u = score_tolerance(ref["scores"], rows, n, tol)
@@ -143,3 +145,41 @@ def test_ragged_paged(mode, tol):
     wl = gen.Workload("rp", 32, 1, 8, 2, 128, 16, gen.POOL_MAX, 7, 0,
                       seq_lens=(300, 40, 2050, 129), budget_frac=0.1, page_size=16)
     check_layer(wl, gen.make_layer(wl), mode, tol)
+
+
+@pytest.mark.parametrize("mode,tol", MODES)
+@pytest.mark.parametrize("ratio,smin", [(0.5, 16), (0.25, 0), (0.3, 64)])
+def test_span_cap_through_the_fused_call(mode, tol, ratio, smin):
+    """Protected tokens limited to B_span = min(B, max(B_min, floor(rho * B))) (Section 4.4, "Span
+    selection under budget"): more protected tokens than the cap, the attention scores fill the rest."""
+    from dataclasses import replace
+    wl = replace(gen.workloads()["tiny"], span_ratio=ratio, span_min=smin, budget=200)
+    check_layer(wl, gen.make_layer(wl, layer=7), mode, tol)
+
+
+@pytest.mark.parametrize("mode,tol", MODES)
+def test_span_cap_ragged_paged_and_chunked(mode, tol):
+    wl = gen.Workload("rpcap", 34, 1, 8, 2, 128, 16, gen.POOL_AVG, 5, 0,
+                      seq_lens=(700, 40, 2050, 129), budget_frac=0.3, page_size=16,
+                      span_ratio=0.5, span_min=16)
+    check_layer(wl, gen.make_layer(wl), mode, tol)
+    wl = gen.Workload("chcap", 35, 1, 8, 2, 128, 32, gen.POOL_NONE, 1, 300, n=3003, chunk_size=10,
+                      span_ratio=0.5, span_min=16)
+    check_layer(wl, gen.make_layer(wl), mode, tol)
+
+
+def test_more_items_than_a_cluster_holds():
+    """A sequence of more than 131072 items: the fused call and cc_topk_select take the
+    single-CTA selection kernel and the stand-alone pooling kernel instead of the cluster kernel."""
+    wl = gen.Workload("long", 36, 1, 2, 1, 128, 8, gen.POOL_MAX, 7, 9000, n=140000)
+    x = gen.make_layer(wl)
+    check_layer(wl, x, cc.CC_MODE_BF16, 2e-3)
+    # selection stage alone on the oracle's fp32 stage values: bit for bit
+    from test_gpu_stages import run_select
+    rng = np.random.Generator(np.random.PCG64(9))
+    u = (np.abs(rng.standard_normal((1, wl.n))) * 1e-3).astype(np.float32)
+    fused = orc.pool_scores(u, orc.POOL_MAX, 7, dtype=np.float32)
+    idx, count = run_select(fused, x.prior, wl.n, wl.budget, wl.force_threshold, 0.5, 16)
+    ref = orc.select_tokens(fused[0], x.prior, wl.n, wl.budget, wl.force_threshold, 0.5, 16)
+    assert count[0] == len(ref) == wl.budget
+    np.testing.assert_array_equal(idx[0, :len(ref)], ref)

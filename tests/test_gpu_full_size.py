@@ -15,10 +15,7 @@ pytestmark = pytest.mark.gpu
 
 @pytest.mark.parametrize("name", ["llama3_8b", "qwen25_coder_7b", "chunk10", "paper_avg5_w128"])
 def test_benchmark_workload_full_size(name):
-    wl = gen.workloads()[name]
-    if wl.span_ratio:
-        from dataclasses import replace
-        wl = replace(wl, span_ratio=0.0)      # check_layer's tolerance band assumes uncapped protection
+    wl = gen.workloads()[name]      # paper_avg5_w128 runs with its span cap (0.5, minimum 16) on
     check_layer(wl, gen.make_layer(wl, layer=1), cc.CC_MODE_BF16, 2e-3)
 
 

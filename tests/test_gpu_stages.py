@@ -243,6 +243,59 @@ def test_compact_paged():
     np.testing.assert_array_equal(after_k[untouched_rows], before_k[untouched_rows])
 
 
+def test_page_ids_outside_the_pool_are_skipped_and_flagged():
+    """A page id equal to pool_pages (one past the pool) in the page table or in the list of fresh
+    pages: the kernels skip the access and record CC_ERR_DEVICE_FLAG.  The pool tensors carry
+    guard pages behind the pool, which must stay untouched."""
+    wl = gen.Workload("p", 12, 1, 4, 2, 128, 8, gen.POOL_MAX, 3, 0, seq_lens=(100, 37),
+                      budget_frac=0.25, page_size=16)
+    x = gen.make_layer(wl)
+    buds = wl.budgets
+    b_tot = sum(buds)
+    idx = np.full((wl.n_heads_kv, b_tot), -1, np.int32)
+    off = 0
+    for n, b in zip(wl.lens, buds):
+        idx[:, off:off + b] = np.arange(b)[None, :]
+        off += b
+    guard_pages = 4
+    hkv = wl.n_heads_kv
+
+    def padded(bits):
+        pad = np.full((guard_pages * 16, hkv, 128), 0x7FC0, np.uint16)
+        return bf16_dev(np.concatenate([bits, pad]))
+
+    stride = max((b + 15) // 16 for b in buds) + 2
+    for where in ("page_table", "free_pages"):
+        table = x.page_table.copy()
+        free = x.free_pages.copy()
+        if where == "page_table":
+            table[0, 0] = x.pool_pages              # tokens 0..15 of sequence 0 point past the pool
+        else:
+            free[0] = x.pool_pages
+        pt = torch.from_numpy(table).cuda()
+        d = desc_for(wl, cc.CC_MODE_FP32, page_table=pt, out_pt_stride=stride, pool_pages=x.pool_pages)
+        k_pool, v_pool = padded(x.k), padded(x.v)
+        out_pt = torch.full((len(buds), stride), -7, dtype=torch.int32, device="cuda")
+        cc.cc_compact_kv(ctx(), d, k_pool, v_pool, torch.from_numpy(idx).cuda(), k_pool, v_pool,
+                         torch.from_numpy(free).cuda(), out_pt)
+        assert ctx().poll() == cc.CC_ERR_DEVICE_FLAG
+        assert (bits_host(k_pool)[x.pool_pages * 16:] == 0x7FC0).all()
+        assert (bits_host(v_pool)[x.pool_pages * 16:] == 0x7FC0).all()
+        if where == "free_pages":
+            assert out_pt.cpu().numpy()[0, 0] == -1       # the bad page is not published
+    # the fp32 score kernel reads K through the same table
+    table = x.page_table.copy()
+    table[1, 1] = x.pool_pages
+    pt = torch.from_numpy(table).cuda()
+    d = desc_for(wl, cc.CC_MODE_FP32, page_table=pt, out_pt_stride=stride, pool_pages=x.pool_pages)
+    scores = torch.zeros((hkv, sum(wl.lens)), device="cuda")
+    cc.cc_score_window(ctx(), d, bf16_dev(x.q_win), padded(x.k), scores)
+    assert ctx().poll() == cc.CC_ERR_DEVICE_FLAG
+    d = desc_for(wl, cc.CC_MODE_BF16, page_table=pt, out_pt_stride=stride, pool_pages=x.pool_pages)
+    cc.cc_score_window(ctx(), d, bf16_dev(x.q_win), padded(x.k), scores)
+    assert ctx().poll() == cc.CC_ERR_DEVICE_FLAG
+
+
 # ------------------------------------------------------------------ argument checks
 def test_descriptor_validation():
     c = ctx()

@@ -307,6 +307,65 @@ def test_compress_sequence_invariants_on_tiny_workload():
         assert np.all(res["pooled"][h] >= res["scores"][h])             # max-pool dominates
 
 
+def _compose_by_hand(q_bits, k_bits, prior, hkv, pool_kind, pool_size, budget, alpha, beta, theta,
+                     span_ratio, span_min, chunk):
+    """The whole path written out from the stage functions that the tests above pin one by one
+    (scalar loops for the chunk level and the fusion, so that no helper of compress_sequence's
+    wiring is reused)."""
+    u, _ = orc.window_scores(orc.bf16_bits_to_f64(q_bits), orc.bf16_bits_to_f64(k_bits), hkv)
+    n = u.shape[1]
+    out = []
+    for h in range(hkv):
+        if chunk > 1:
+            m = (n + chunk - 1) // chunk
+            item = [sum(u[h, c * chunk:min(n, (c + 1) * chunk)]) for c in range(m)]
+            item_p = [max(prior[c * chunk:min(n, (c + 1) * chunk)]) for c in range(m)]
+        else:
+            item = list(orc.pool_scores(u[h:h + 1], pool_kind, pool_size)[0])
+            item_p = list(prior)
+        fused = [alpha * a + beta * p for a, p in zip(item, item_p)]
+        out.append(orc.select_tokens(np.array(fused), np.array(item_p, np.float32), n, budget,
+                                     theta, span_ratio, span_min, chunk))
+    return out
+
+
+@pytest.mark.parametrize("chunk,span_ratio,span_min,beta", [(1, 0.5, 2, 0.0), (5, 0.0, 0, 0.3),
+                                                          (5, 0.5, 2, 0.0), (4, 0.4, 5, 0.7)])
+def test_compress_sequence_wiring_with_chunks_and_span_cap(chunk, span_ratio, span_min, beta):
+    """30 tokens; priors of several sizes placed so that a chunk's prior (its maximum) differs
+    from the prior of its first token, and more protected tokens than the span budget: taking
+    the token prior for the chunk prior, dropping the cap arguments or swapping alpha and beta
+    changes the retained set."""
+    n, hq, hkv, w, budget = 30, 4, 2, 3, 12
+    q, k, v = gen.small_case(77, n, w, hq, hkv)
+    prior = np.zeros(n, np.float32)
+    prior[[3, 7, 8, 14, 21, 22, 23, 29]] = [0.9, 0.6, 1.0, 0.8, 0.7, 0.55, 0.95, 0.65]
+    res = orc.compress_sequence(q, k, v, prior, hkv, orc.POOL_MAX if chunk == 1 else orc.POOL_NONE,
+                                3 if chunk == 1 else 1, budget, 1.0, beta, 0.5, span_ratio,
+                                span_min, chunk)
+    ref = _compose_by_hand(q, k, prior, hkv, orc.POOL_MAX if chunk == 1 else orc.POOL_NONE,
+                           3 if chunk == 1 else 1, budget, 1.0, beta, 0.5, span_ratio, span_min, chunk)
+    for h in range(hkv):
+        assert len(res["idx"][h]) == budget
+        assert res["idx"][h].tolist() == ref[h].tolist()
+        np.testing.assert_array_equal(res["k_out"][h], k[res["idx"][h], h])
+    if chunk > 1:
+        # the chunk prior is the maximum over the chunk, not the prior of its first token
+        m = (n + chunk - 1) // chunk
+        assert res["item_prior"].tolist() == [float(prior[c * chunk:(c + 1) * chunk].max()) for c in range(m)]
+        assert any(res["item_prior"][c] != prior[c * chunk] for c in range(m))
+    if span_ratio > 0:
+        cap = orc.span_budget(budget, span_ratio, span_min)
+        lens = orc.chunk_lengths(n, chunk)
+        prot = orc.protected_items(res["item_prior"], lens, budget, 0.5, span_ratio, span_min)
+        uncapped = orc.protected_items(res["item_prior"], lens, budget, 0.5)
+        assert lens[prot].sum() <= cap < lens[uncapped].sum()      # the cap is what limits them
+        # the retained set differs from what the uncapped rule would keep
+        other = orc.compress_sequence(q, k, v, prior, hkv, orc.POOL_MAX if chunk == 1 else orc.POOL_NONE,
+                                      3 if chunk == 1 else 1, budget, 1.0, beta, 0.5, 0.0, 0, chunk)
+        assert any(other["idx"][h].tolist() != res["idx"][h].tolist() for h in range(hkv))
+
+
 def test_workload_recipe_statistics():
     wls = gen.workloads()
     p, lab = gen.structural_prior(1, 200000)
