@@ -6,15 +6,22 @@ on one layer of the workload.  The metric is prefix tokens compressed per second
 with N GPUs every rank compresses its own layer stream (weak scaling, no data-path
 collective) and the value is the sum over ranks.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama3_8b] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload ragged_paged] [--impl reference]
 
-Prints one JSON line (rank 0).  ``--impl reference`` times the CPU oracle instead.
+Prints one JSON line (rank 0).  The headline figures are those of ``--workload`` (default: the
+ragged paged batch, the largest configuration); ``workloads`` in the same line holds the fused
+step and its stages for every configuration, with K/V cold and warm in L2.
+``--impl reference`` times the CPU oracle instead.  With ``--gpus N`` and no torchrun
+environment the script starts the N ranks itself.
 """
 from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -26,7 +33,21 @@ sys.path.insert(0, ROOT)
 
 METRIC = "prefix tokens compressed/sec per layer (score+prior+topk+gather)"
 UNIT = "tokens/s/layer"
-N_LAYER_SETS = 4          # distinct K/V sets cycled through so that no step finds its keys in L2
+L2_BYTES = 126e6
+TIMED_BLOCKS = 50         # the block of --steps steps is timed this many times; the median counts
+
+# Exponentials per clock per SM of the score kernel's inner loop (special-function unit plus the
+# packed-FMA polynomial, 7 pairs in 16 on the FMA pipe), measured on a B200 with the loop alone on
+# 16 warps per SM: values held in registers / values read from tensor memory as the kernel does.
+# Source: profiles/exp_throughput_microbenchmark.md.
+EXP_PER_CLK_SM_REGISTERS = 22.6
+EXP_PER_CLK_SM_TMEM = 17.6
+SM_COUNT = 148
+
+# DRAM bytes (read + write) of the two launches of the score stage, per workload, from the ncu
+# captures summarised under profiles/ (counters taken on the kernel as it stands in this tree):
+# "live" = caches left alone between the launches, "flushed" = ncu's default cache flush.
+SCORE_TRAFFIC_BYTES = {}
 
 
 def load_peaks():
@@ -42,8 +63,9 @@ def load_peaks():
 
 
 def algorithmic_work(wl):
-    """Bytes and flops one layer needs on paper: K read once, Q, prior, the gathered K/V rows
-    read and written once, the index lists; 2*w*G*d flops per (key, KV head)."""
+    """Bytes, flops and exponentials one layer needs on paper: K read once, Q, prior, the
+    gathered K/V rows read and written once, the index lists; 2*w*G*d flops and w*G
+    exponentials per (key, KV head)."""
     d, hkv, hq, w = wl.head_dim, wl.n_heads_kv, wl.n_heads_q, wl.window
     n_tot = sum(wl.lens)
     keep = sum(min(b, n) for b, n in zip(wl.budgets, wl.lens))
@@ -55,7 +77,25 @@ def algorithmic_work(wl):
     bytes_total = k_bytes + q_bytes + 4 * n_tot + gather_bytes
     flops = 2.0 * w * wl.group * d * n_tot * hkv
     return {"bytes": float(bytes_total), "flops": flops, "score_bytes": float(score_bytes),
-            "gather_bytes": float(gather_bytes), "tokens": n_tot}
+            "gather_bytes": float(gather_bytes), "tokens": n_tot,
+            "exps": float(w * wl.group * n_tot * hkv)}
+
+
+def roofline_of(work, peaks, seconds, clock_mhz=None):
+    """Path roofline: the larger of bytes / HBM bandwidth and flops / bf16 tensor peak, against
+    the measured duration; the exponential ceiling as a third number beside them."""
+    t_bytes = work["bytes"] / (peaks["hbm_gbs"] * 1e9)
+    t_flops = work["flops"] / (peaks["bf16_tflops"] * 1e12)
+    t_roof = max(t_bytes, t_flops)
+    out = {"bound": "hbm" if t_bytes >= t_flops else "tensor", "t_roof_us": t_roof * 1e6,
+           "t_bytes_us": t_bytes * 1e6, "t_flops_us": t_flops * 1e6, "t_path_us": seconds * 1e6,
+           "frac": t_roof / seconds}
+    if clock_mhz:
+        # both passes of the score stage evaluate every exponential once
+        per_s = EXP_PER_CLK_SM_REGISTERS * SM_COUNT * clock_mhz * 1e6
+        out["exp_bound_us"] = 2.0 * work["exps"] / per_s * 1e6
+        out["exp_bound_us_tmem_reads"] = 2.0 * work["exps"] / (EXP_PER_CLK_SM_TMEM * SM_COUNT * clock_mhz * 1e6) * 1e6
+    return out
 
 
 class ClockSampler(threading.Thread):
@@ -64,6 +104,7 @@ class ClockSampler(threading.Thread):
     def __init__(self, index: int):
         super().__init__(daemon=True)
         self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self.power = []
         self._stop_evt = threading.Event()
         self.ok = False
         try:
@@ -90,6 +131,10 @@ class ClockSampler(threading.Thread):
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
                 try:
+                    self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+                except Exception:
+                    pass
+                try:
                     mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
                 except Exception:
                     mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
@@ -105,7 +150,8 @@ class ClockSampler(threading.Thread):
         self.join(timeout=2)
         med = float(np.median(self.samples)) if self.samples else None
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+                "samples": len(self.samples),
+                "power_w_max": max(self.power) if self.power else None}
 
 
 # ----------------------------------------------------------------------------- CPU oracle arm
@@ -114,7 +160,7 @@ _ORACLE_INPUTS = {}
 
 def oracle_throughput(wl, budget_s: float):
     """Times the oracle (as it stands) on a bounded sample of one layer: a subset of the KV
-    heads, all keys, whole path.  Returns tokens/s/layer scaled to all heads."""
+    heads, all keys of sequence 0, whole path.  Returns tokens/s/layer scaled to all heads."""
     from oracle import codecomp_oracle as orc
     from paper_2604_10235_b200 import inputs as gen
     if wl.name not in _ORACLE_INPUTS:
@@ -173,7 +219,7 @@ def run_reference(args, wl):
             "n_gpus": args.gpus, "steps": len(times), "warmup": args.warmup,
             "ms_per_step": 1e3 * sum(wl.lens) / value, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": wl.name, "note": "CPU oracle, NumPy fp64, host cores"},
+            "config": bench_config(wl, None, None),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"], "kind": "oracle",
                              "sample": last["sample"]},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -181,14 +227,153 @@ def run_reference(args, wl):
     print(json.dumps(line), flush=True)
 
 
+def bench_config(wl, n_sets, set_bytes):
+    """The ``config`` object of the JSON line: the same keys for both arms."""
+    cfg = {"workload": wl.name, "n": list(wl.lens), "heads_q": wl.n_heads_q,
+           "heads_kv": wl.n_heads_kv, "window": wl.window, "pool": [wl.pool_kind, wl.pool_size],
+           "budget": list(wl.budgets), "chunk": wl.chunk_size, "page_size": wl.page_size}
+    if n_sets is not None:
+        cfg["layers_cycled"] = n_sets
+        cfg["launch"] = f"CUDA graph of {n_sets} fused steps, replayed"
+        cfg["l2"] = (f"inputs larger than L2: {n_sets} layer sets of {set_bytes / 1e6:.0f} MB cycled, "
+                     f"no set reused within {(n_sets - 1) * set_bytes / 1e6:.0f} MB of traffic")
+    return cfg
+
+
 # ----------------------------------------------------------------------------- CUDA arm
+def bench_workloads():
+    """Every configuration of the benchmark table, in the order reported."""
+    from paper_2604_10235_b200 import inputs as gen
+    w = gen.workloads()
+    q = w["qwen25_coder_7b"]
+    table = [w["tiny"], w["llama3_8b"]]
+    table += [gen.qwen_variant(q, b, "15") for b in (1024, 4096, 8192)]
+    table += [w["chunk10"], w["ragged_paged"], w["paper_avg5_w128"]]
+    return {x.name: x for x in table}
+
+
+def sets_for(wl) -> int:
+    """Layer sets to cycle so that a set is not found in L2 when its turn comes again."""
+    row = wl.head_dim * 2
+    set_bytes = 2 * sum(wl.lens) * wl.n_heads_kv * row
+    return int(min(100, max(2, math.ceil(512e6 / max(set_bytes, 1)))))
+
+
+class WorkloadRun:
+    """Device-resident inputs of one workload and the graphs that replay its calls."""
+
+    def __init__(self, ctx, wl, rank: int, pinned: bool):
+        import torch
+        from paper_2604_10235_b200 import inputs as gen
+        from paper_2604_10235_b200 import sharding
+        from paper_2604_10235_b200.api import LayerCompressor, to_bf16
+        self.torch, self.ctx, self.wl = torch, ctx, wl
+        self.n_sets = sets_for(wl)
+        layers = sharding.rank_layers(rank, self.n_sets)
+        layout0 = gen.make_layer(wl, layer=layers[0]) if wl.page_size else None
+        self.comp = LayerCompressor(ctx, wl, layout=layout0)
+        self.dev_sets, self.host_sets = [], []
+        for i, layer in enumerate(layers):
+            x = layout0 if (i == 0 and layout0 is not None) else gen.make_layer(wl, layer=layer)
+            if rank == 0 and i == 0:
+                _ORACLE_INPUTS.setdefault(wl.name, x)     # layer 0: what the CPU baseline runs on
+            if wl.page_size and i > 0:
+                gen.repage(x, layout0)          # every layer set uses the page layout of the first
+            hs = (to_bf16(x.q_win, "cpu", pin=pinned), to_bf16(x.k, "cpu", pin=pinned),
+                  to_bf16(x.v, "cpu", pin=pinned),
+                  torch.from_numpy(x.prior).pin_memory() if pinned else torch.from_numpy(x.prior))
+            if pinned and i < 2:
+                self.host_sets.append(hs)
+            self.dev_sets.append(tuple(t.cuda() for t in hs))
+        self.set_bytes = sum(t.numel() * t.element_size() for t in self.dev_sets[0])
+        self.side = torch.cuda.Stream()
+
+    def capture(self, fn, sets):
+        """One CUDA graph that calls fn on each of the given layer sets."""
+        torch = self.torch
+        for s in sets:
+            fn(*s)
+        torch.cuda.synchronize()
+        self.side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(self.side):
+            with torch.cuda.graph(graph, stream=self.side):
+                for s in sets:
+                    fn(*s)
+        torch.cuda.current_stream().wait_stream(self.side)
+        graph.replay()
+        torch.cuda.synchronize()
+        return graph
+
+    def time_graph(self, graph, calls_per_replay, total_calls=200):
+        torch = self.torch
+        reps = max(1, total_calls // calls_per_replay)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / (reps * calls_per_replay)
+
+    def stage_fns(self):
+        from paper_2604_10235_b200 import binding as cc
+        torch, comp, wl, ctx = self.torch, self.comp, self.wl, self.ctx
+        d = comp.desc
+        scores = torch.empty((wl.n_heads_kv, d.n_tot), device="cuda")
+        fused = torch.empty((wl.n_heads_kv, d.m_tot), device="cuda")
+        self.str_score = torch.empty((len(wl.lens), wl.n_heads_kv), device="cuda")
+
+        def score(q, k, v, p):
+            cc.cc_score_window(ctx, d, q, k, scores, None, ws=comp.ws)
+
+        def fuse_pool(q, k, v, p):
+            cc.cc_fuse_prior_pool(ctx, d, scores, p, fused)
+
+        def select(q, k, v, p):
+            cc.cc_topk_select(ctx, d, fused, p, comp.idx, comp.count, ws=comp.ws)
+
+        def compact(q, k, v, p):
+            if comp.paged:
+                cc.cc_compact_kv(ctx, d, k, v, comp.idx, k, v, comp.free_pages, comp.out_page_table)
+            else:
+                cc.cc_compact_kv(ctx, d, k, v, comp.idx, comp.k_out, comp.v_out)
+
+        def str_score(q, k, v, p):
+            # not part of a step: the retained fraction of the structurally critical tokens
+            cc.cc_structural_score(ctx, d, comp.idx, p, wl.force_threshold, self.str_score)
+
+        return {"score": score, "fuse_pool": fuse_pool, "select": select, "compact": compact,
+                "str_score_diagnostic": str_score}
+
+    def table_entry(self, peaks, clock_mhz):
+        """Fused step cold and warm in L2, the stages on their own (cold), the path roofline."""
+        work = algorithmic_work(self.wl)
+        cold = self.capture(self.comp.run_device, self.dev_sets)
+        ms_cold = self.time_graph(cold, self.n_sets)
+        warm = self.capture(self.comp.run_device, [self.dev_sets[0]] * 4)
+        ms_warm = self.time_graph(warm, 4)
+        stage_us = {}
+        for name, fn in self.stage_fns().items():
+            g = self.capture(fn, self.dev_sets)
+            stage_us[name] = self.time_graph(g, self.n_sets) * 1e3
+        if self.ctx.poll() != 0:
+            raise RuntimeError(f"device status after the runs of {self.wl.name}")
+        cold_l2 = self.n_sets * self.set_bytes > 1.5 * L2_BYTES
+        return {"ms_per_step": ms_cold, "ms_per_step_warm_l2": ms_warm,
+                "tokens_per_s": work["tokens"] / (ms_cold * 1e-3), "stage_us": stage_us,
+                "path_roofline": roofline_of(work, peaks, ms_cold * 1e-3, clock_mhz),
+                "path_roofline_warm_l2": roofline_of(work, peaks, ms_warm * 1e-3, clock_mhz),
+                "layer_sets": self.n_sets, "set_mb": self.set_bytes / 1e6,
+                "cold_l2": bool(cold_l2),
+                "str_score_mean": float(self.str_score.mean().item())}
+
+
 def run_ours(args, wl):
     import torch
     import torch.distributed as dist
     from paper_2604_10235_b200 import binding as cc
-    from paper_2604_10235_b200 import inputs as gen
     from paper_2604_10235_b200 import sharding
-    from paper_2604_10235_b200.api import LayerCompressor, to_bf16
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -199,23 +384,12 @@ def run_ours(args, wl):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     ctx = cc.Context(local)
-    layers = sharding.rank_layers(rank, N_LAYER_SETS)
-    layout0 = gen.make_layer(wl, layer=layers[0]) if wl.page_size else None
-    comp = LayerCompressor(ctx, wl, layout=layout0)
-    work = algorithmic_work(wl)
     peaks = load_peaks()
+    work = algorithmic_work(wl)
 
-    # inputs: N_LAYER_SETS layers, resident in HBM before timing, plus pinned host copies
-    dev_sets, host_sets = [], []
-    for i, layer in enumerate(layers):
-        x = gen.make_layer(wl, layer=layer)
-        if wl.page_size and i > 0:
-            gen.repage(x, layout0)          # every layer set uses the page layout of the first
-        hs = (to_bf16(x.q_win, "cpu", pin=True), to_bf16(x.k, "cpu", pin=True),
-              to_bf16(x.v, "cpu", pin=True), torch.from_numpy(x.prior).pin_memory())
-        host_sets.append(hs)
-        dev_sets.append(tuple(t.cuda() for t in hs))
-    set_bytes = sum(t.numel() * t.element_size() for t in dev_sets[0])
+    # inputs: layer sets resident in HBM before timing, plus pinned host copies of two of them
+    run = WorkloadRun(ctx, wl, rank, pinned=True)
+    comp, n_sets = run.comp, run.n_sets
 
     def barrier():
         sharding.barrier(world)
@@ -224,141 +398,120 @@ def run_ours(args, wl):
     def max_over_ranks(ms: float) -> float:
         return sharding.max_over_ranks(ms, world, "cuda")
 
-    # ---- device-resident timing: the fused call on each of the layer sets is captured once in
-    # a CUDA graph (one replay = N_LAYER_SETS steps), so the timed region holds kernel time and
-    # launch dependencies, not the Python binding's host time between calls
+    # ---- device-resident timing.  The fused call on each of the layer sets is captured once in
+    # a CUDA graph (one replay = n_sets steps), so the timed region holds kernel time and launch
+    # dependencies, not the Python binding's host time between calls.  A block of exactly
+    # --steps steps is timed TIMED_BLOCKS times back to back (so the figure is the sustained one
+    # and the clock sampler sees the load); the median block counts.
     for i in range(args.warmup):
-        comp.run_device(*dev_sets[i % N_LAYER_SETS])
+        comp.run_device(*run.dev_sets[i % n_sets])
     assert ctx.poll() == 0
-    side = torch.cuda.Stream()
-    side.wait_stream(torch.cuda.current_stream())
-    graph = torch.cuda.CUDAGraph()
-    with torch.cuda.stream(side):
-        with torch.cuda.graph(graph, stream=side):
-            for j in range(N_LAYER_SETS):
-                comp.run_device(*dev_sets[j])
-    torch.cuda.current_stream().wait_stream(side)
-    graph.replay()
-    n_replays, n_rest = divmod(args.steps, N_LAYER_SETS)
+    graph = run.capture(comp.run_device, run.dev_sets)
+    n_replays, n_rest = divmod(args.steps, n_sets)
     sampler = ClockSampler(local)
+    events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+              for _ in range(TIMED_BLOCKS)]
     barrier()
     sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(n_replays):
-        graph.replay()
-    for j in range(n_rest):
-        comp.run_device(*dev_sets[j])
-    e1.record()
+    for e0, e1 in events:
+        e0.record()
+        for _ in range(n_replays):
+            graph.replay()
+        for j in range(n_rest):
+            comp.run_device(*run.dev_sets[j])
+        e1.record()
     barrier()
     clocks = sampler.stop()
-    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    block_ms = sorted(e0.elapsed_time(e1) for e0, e1 in events)
+    ms_total = max_over_ranks(block_ms[len(block_ms) // 2])
     status = ctx.poll()
     if status != 0:
         raise RuntimeError(f"device status {status} after the timed region")
     ms_step = ms_total / args.steps
     value = sharding.job_throughput(work["tokens"], world, ms_step)
+    clock_mhz = clocks["sm_mhz"] or 1965.0
 
-    # ---- per-stage durations: each stage entry point captured the same way and replayed
-    d = comp.desc
-    scores = torch.empty((wl.n_heads_kv, d.n_tot), device="cuda")
-    fused = torch.empty((wl.n_heads_kv, d.m_tot), device="cuda")
-
-    def stage_call(k, q_d, k_d, v_d, p_d):
-        if k == 0:
-            cc.cc_score_window(ctx, d, q_d, k_d, scores, None, ws=comp.ws)
-        elif k == 1:
-            cc.cc_fuse_prior_pool(ctx, d, scores, p_d, fused)
-        elif k == 2:
-            cc.cc_topk_select(ctx, d, fused, p_d, comp.idx, comp.count, ws=comp.ws)
-        elif k == 3:
-            if comp.paged:
-                cc.cc_compact_kv(ctx, d, k_d, v_d, comp.idx, k_d, v_d, comp.free_pages,
-                                 comp.out_page_table)
-            else:
-                cc.cc_compact_kv(ctx, d, k_d, v_d, comp.idx, comp.k_out, comp.v_out)
-        else:
-            # not part of a step: the retained fraction of the structurally critical tokens
-            cc.cc_structural_score(ctx, d, comp.idx, p_d, wl.force_threshold, str_score)
-
-    str_score = torch.empty((len(wl.lens), wl.n_heads_kv), device="cuda")
-    stage_ms = np.zeros(5)
-    stage_reps = max(1, min(args.steps, 200) // N_LAYER_SETS)
-    for k in range(5):
-        for j in range(N_LAYER_SETS):
-            stage_call(k, *dev_sets[j])
-        torch.cuda.synchronize()
-        side.wait_stream(torch.cuda.current_stream())
-        g_stage = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(side):
-            with torch.cuda.graph(g_stage, stream=side):
-                for j in range(N_LAYER_SETS):
-                    stage_call(k, *dev_sets[j])
-        torch.cuda.current_stream().wait_stream(side)
-        g_stage.replay()
-        torch.cuda.synchronize()
-        e0.record()
-        for _ in range(stage_reps):
-            g_stage.replay()
-        e1.record()
-        torch.cuda.synchronize()
-        stage_ms[k] = e0.elapsed_time(e1) / (stage_reps * N_LAYER_SETS)
-    score_s = stage_ms[0] * 1e-3
-    achieved_tf = work["flops"] / score_s / 1e12
-    t_bytes = work["bytes"] / (peaks["hbm_gbs"] * 1e9)
-    t_flops = work["flops"] / (peaks["bf16_tflops"] * 1e12)
-    t_roof = max(t_bytes, t_flops)
+    # ---- per-stage durations (each stage entry point captured the same way) and the table
+    head = run.table_entry(peaks, clock_mhz)
+    stage_us = head["stage_us"]
+    score_s = stage_us["score"] * 1e-6
+    t_b = work["score_bytes"] / (peaks["hbm_gbs"] * 1e9)
+    t_f = work["flops"] / (peaks["bf16_tflops"] * 1e12)
+    if t_f >= t_b:
+        roof = {"bound": "tensor", "achieved": work["flops"] / score_s / 1e12,
+                "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "peak_source": f"{peaks['source']} bf16 burst"}
+    else:
+        roof = {"bound": "hbm", "achieved": work["score_bytes"] / score_s / 1e9,
+                "peak": peaks["hbm_gbs"], "unit": "GB/s", "peak_source": f"{peaks['source']} copy"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["kernel"] = "score_tc_kernel<1> + score_tc_kernel<2> (the two launches of the score stage)"
+    traffic = SCORE_TRAFFIC_BYTES.get(wl.name, {})
+    roof["traffic"] = traffic.get("live")
+    roof["traffic_caches_flushed"] = traffic.get("flushed")
+    roof["flops_per_launch_pair"] = work["flops"]
+    roof["bytes_per_launch_pair"] = work["score_bytes"]
+    roof["exp_bound_us"] = head["path_roofline"].get("exp_bound_us")
+    roof["time_us"] = stage_us["score"]
 
     # ---- end to end: pinned host inputs in, compacted cache back out, every step
     n_e2e = max(3, min(args.steps, 40))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for i in range(2):
-        comp.run_host(*host_sets[i % N_LAYER_SETS])
+        comp.run_host(*run.host_sets[i % len(run.host_sets)])
     barrier()
     e0.record()
     for i in range(n_e2e):
-        comp.run_host(*host_sets[i % N_LAYER_SETS])
+        comp.run_host(*run.host_sets[i % len(run.host_sets)])
     e1.record()
     barrier()
     ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / n_e2e
     e2e_value = sharding.job_throughput(work["tokens"], world, ms_e2e)
+    h2d, d2h = comp.h2d_bytes, comp.d2h_bytes
+    n_sets_head, set_bytes_head = run.n_sets, run.set_bytes
 
-    aux = chunk_scoring_bandwidth(ctx, peaks) if rank == 0 and world == 1 else None
+    table, aux, cpu = None, None, None
+    if rank == 0 and world == 1 and not args.no_table:
+        table = {wl.name: head}
+        del run, comp, graph
+        torch.cuda.empty_cache()
+        for name, other in bench_workloads().items():
+            if name == wl.name:
+                continue
+            r = WorkloadRun(ctx, other, rank, pinned=False)
+            table[name] = r.table_entry(peaks, clock_mhz)
+            del r
+            torch.cuda.empty_cache()
+        aux = chunk_scoring_bandwidth(ctx, peaks)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = oracle_throughput(wl, 12.0)
+        cpu.pop("seconds", None)
     if rank == 0:
-        cpu = None
-        if world == 1 and not args.no_cpu_baseline:
-            cpu = oracle_throughput(wl, 12.0)
-            cpu.pop("seconds", None)
+        path = roofline_of(work, peaks, ms_step * 1e-3, clock_mhz)
+        path.update({"bytes": work["bytes"], "flops": work["flops"], "exps_per_pass": work["exps"],
+                     "hbm_peak_gbs": peaks["hbm_gbs"], "tensor_peak_tflops": peaks["bf16_tflops"],
+                     "binding_unit": "special-function unit + FMA pipe + instruction issue of the "
+                                     "exponentials (see exp_bound_us), not HBM or the tensor pipe"})
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": wl.name, "layers_cycled": N_LAYER_SETS,
-                       "launch": f"CUDA graph of {N_LAYER_SETS} fused steps, replayed",
-                       "n": list(wl.lens), "heads_q": wl.n_heads_q, "heads_kv": wl.n_heads_kv,
-                       "window": wl.window, "pool": [wl.pool_kind, wl.pool_size],
-                       "budget": list(wl.budgets), "chunk": wl.chunk_size,
-                       "l2": f"inputs larger than L2: {N_LAYER_SETS} layer sets of "
-                             f"{set_bytes / 1e6:.0f} MB cycled, no set reused within "
-                             f"{(N_LAYER_SETS - 1) * set_bytes / 1e6:.0f} MB of traffic"},
-            "roofline": {"bound": "tensor", "kernel": "score_tc_kernel<1> + score_tc_kernel<2> (the two launches of the score stage)",
-                         "achieved": achieved_tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                         "frac": achieved_tf / peaks["bf16_tflops"], "traffic": score_traffic(wl),
-                         "peak_source": f"{peaks['source']} bf16 burst",
-                         "flops_per_launch_pair": work["flops"]},
-            "path_roofline": {"t_roof_us": t_roof * 1e6, "t_bytes_us": t_bytes * 1e6,
-                              "t_flops_us": t_flops * 1e6, "t_path_us": ms_step * 1e3,
-                              "frac": t_roof / (ms_step * 1e-3), "bytes": work["bytes"],
-                              "flops": work["flops"], "hbm_peak_gbs": peaks["hbm_gbs"]},
-            "stage_us": {"score": stage_ms[0] * 1e3, "fuse_pool": stage_ms[1] * 1e3,
-                         "select": stage_ms[2] * 1e3, "compact": stage_ms[3] * 1e3,
-                         "str_score_diagnostic": stage_ms[4] * 1e3},
-            "str_score": [round(float(v), 4) for v in str_score.flatten().tolist()],
+            "config": bench_config(wl, n_sets_head, set_bytes_head),
+            "timing": {"blocks": TIMED_BLOCKS, "block_ms_median": ms_total,
+                       "block_ms_min": block_ms[0], "block_ms_max": block_ms[-1],
+                       "cycles_per_step_at_sampled_clock": ms_step * 1e-3 * clock_mhz * 1e6},
+            "roofline": roof,
+            "path_roofline": path,
+            "stage_us": stage_us,
+            "ms_per_step_warm_l2": head["ms_per_step_warm_l2"],
+            "workloads": table,
             "chunk_scoring": aux,
             "cpu_baseline": cpu,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": comp.h2d_bytes,
-                    "d2h_bytes_per_step": comp.d2h_bytes, "ms_per_step": ms_e2e, "steps": n_e2e},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": n_e2e},
             # per step: score pass 1, score pass 2, pool + fuse + select (one cluster kernel), compact
-            "gpu_launches": 4 * args.steps,
+            "gpu_launches": 4 * args.steps * TIMED_BLOCKS,
+            "gpu_launches_per_step": 4,
             "clocks": clocks,
         }
         print(json.dumps(line), flush=True)
@@ -400,29 +553,63 @@ def chunk_scoring_bandwidth(ctx, peaks):
     return out
 
 
-# DRAM bytes (read + write) of one launch pair of the score stage, from the ncu capture that
-# is summarised under profiles/ (llama3_8b: 67.67 + 0.81 MB for pass 1,
-# 68.00 + 1.44 MB for pass 2).  The counters were taken on the kernel as it stands in this tree;
-# other workloads have no capture and report null.
-SCORE_TRAFFIC_BYTES = {"llama3_8b": 137.93e6}
+# ----------------------------------------------------------------------------- multi-process launch
+def run_stub(args):
+    """The multi-rank skeleton of run_ours without a GPU: gloo ranks, a barrier, a timed block of
+    trivial host steps, the max over ranks, one JSON line from rank 0.  Used by the CPU test of
+    the launcher."""
+    import torch.distributed as dist
+    from paper_2604_10235_b200 import sharding
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    layers = sharding.rank_layers(rank, 2)
+    sharding.barrier(world)
+    t0 = time.perf_counter()
+    acc = 0
+    for i in range(args.steps):
+        acc += sum(layers) + i
+    ms = sharding.max_over_ranks((time.perf_counter() - t0) * 1e3 + 1.0 + rank, world)
+    if rank == 0:
+        print(json.dumps({"impl": "stub", "n_gpus": world, "steps": args.steps,
+                          "ms_per_step": ms / max(1, args.steps),
+                          "value": sharding.job_throughput(1000, world, ms / max(1, args.steps))}),
+              flush=True)
+    if world > 1:
+        dist.destroy_process_group()
 
 
-def score_traffic(wl):
-    return SCORE_TRAFFIC_BYTES.get(wl.name)
+def launch_ranks(args, argv) -> int:
+    """Starts --gpus ranks of this script on this node (one per device) through torch's launcher
+    and passes their output through; rank 0 prints the JSON line."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+           f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1", "--master-port", str(port),
+           os.path.abspath(__file__)] + argv
+    return subprocess.call(cmd)
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="llama3_8b")
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "stub"])
+    ap.add_argument("--workload", default="ragged_paged")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-table", action="store_true", help="skip the table of the other workloads")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        sys.exit(launch_ranks(args, sys.argv[1:]))
+    if args.impl == "stub":
+        run_stub(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     from paper_2604_10235_b200 import inputs as gen
-    wl = gen.workloads()[args.workload]
+    wl = {**gen.workloads(), **bench_workloads()}[args.workload]
     if args.impl == "reference":
         run_reference(args, wl)
     else:

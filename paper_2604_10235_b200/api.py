@@ -11,22 +11,60 @@ from typing import Dict, Optional
 import numpy as np
 import torch
 
+from dataclasses import dataclass, fields
+from typing import Tuple
+
 from . import binding as cc
-from . import inputs as gen
 
 
-def desc_from_workload(wl: gen.Workload, mode: int = cc.CC_MODE_BF16,
-                       page_table: Optional[torch.Tensor] = None, pool_pages: int = 0,
-                       out_pt_stride: int = 0) -> cc.Desc:
+@dataclass(frozen=True)
+class LayerSpec:
+    """Geometry and settings of one layer's compression step (what ``cc_layer_desc`` holds,
+    minus pointers): heads, window, pooling, prior fusion, protection and its cap, the
+    sequences of the batch with their budgets, and the K/V layout."""
+
+    n_heads_q: int
+    n_heads_kv: int
+    window: int
+    lens: Tuple[int, ...]                 # tokens per sequence
+    budgets: Tuple[int, ...]              # tokens kept per KV head, per sequence
+    head_dim: int = 128
+    pool_kind: int = cc.CC_POOL_MAX
+    pool_size: int = 7
+    chunk_size: int = 1
+    alpha: float = 1.0
+    beta: float = 0.0
+    force_threshold: float = float("inf")
+    span_ratio: float = 0.0
+    span_min: int = 0
+    page_size: int = 0                    # 0 = contiguous K/V
+    causal: bool = False
+
+    @classmethod
+    def like(cls, obj) -> "LayerSpec":
+        """A spec with the values of the equally named attributes of ``obj`` (any object that
+        describes a layer: a benchmark workload, a model configuration, ...)."""
+        kw = {f.name: getattr(obj, f.name) for f in fields(cls) if hasattr(obj, f.name)}
+        kw["lens"], kw["budgets"] = tuple(kw["lens"]), tuple(kw["budgets"])
+        return cls(**kw)
+
+    @property
+    def group(self) -> int:
+        return self.n_heads_q // self.n_heads_kv
+
+
+def desc_from_spec(wl: LayerSpec, mode: int = cc.CC_MODE_BF16,
+                   page_table: Optional[torch.Tensor] = None, pool_pages: int = 0,
+                   out_pt_stride: int = 0) -> cc.Desc:
     kw = dict(head_dim=wl.head_dim, compute_mode=mode, pool_kind=wl.pool_kind,
               pool_size=wl.pool_size, chunk_size=wl.chunk_size, alpha=wl.alpha, beta=wl.beta,
               force_threshold=wl.force_threshold, span_ratio=wl.span_ratio, span_min=wl.span_min,
               page_size=wl.page_size, page_table=page_table, pool_pages=pool_pages,
               out_page_table_stride=out_pt_stride, causal=wl.causal)
-    if wl.seq_lens:
+    if len(wl.lens) > 1 or wl.page_size:
         return cc.Desc(wl.n_heads_q, wl.n_heads_kv, wl.window, seq_lens=wl.lens,
                        budgets=wl.budgets, **kw)
-    return cc.Desc(wl.n_heads_q, wl.n_heads_kv, wl.window, n=wl.n, budget=wl.budget, **kw)
+    return cc.Desc(wl.n_heads_q, wl.n_heads_kv, wl.window, n=wl.lens[0], budget=wl.budgets[0], **kw)
 
 
 def to_bf16(bits: np.ndarray, device: str = "cuda", pin: bool = False) -> torch.Tensor:
@@ -39,13 +77,14 @@ def to_bf16(bits: np.ndarray, device: str = "cuda", pin: bool = False) -> torch.
 class LayerCompressor:
     """Pre-allocated state for repeated ``cc_compress_layer`` calls on one geometry.
 
-    Contiguous K/V: the compacted cache lands in ``k_out`` / ``v_out``.  Paged K/V
-    (``wl.page_size > 0``): ``layout`` supplies the page table, the list of fresh pages and
-    the pool size (a ``LayerInputs`` of the workload); the retained rows are written into
-    fresh pages of the same pool and ``out_page_table`` names them."""
+    ``spec`` is a ``LayerSpec`` (or any object with its attributes).  Contiguous K/V: the
+    compacted cache lands in ``k_out`` / ``v_out``.  Paged K/V (``spec.page_size > 0``):
+    ``layout`` supplies ``page_table`` [S][pages] (int32, numpy), ``free_pages`` (fresh page
+    ids, int32, numpy) and ``pool_pages``; the retained rows are written into fresh pages of the
+    same pool and ``out_page_table`` names them."""
 
-    def __init__(self, ctx: cc.Context, wl: gen.Workload, mode: int = cc.CC_MODE_BF16,
-                 layout: Optional[gen.LayerInputs] = None):
+    def __init__(self, ctx: cc.Context, spec, mode: int = cc.CC_MODE_BF16, layout=None):
+        wl = spec if isinstance(spec, LayerSpec) else LayerSpec.like(spec)
         self.ctx, self.wl = ctx, wl
         dev = f"cuda:{ctx.device}"
         self.paged = wl.page_size > 0
@@ -53,19 +92,19 @@ class LayerCompressor:
         bf = torch.bfloat16
         if self.paged:
             if layout is None or layout.page_table is None:
-                raise ValueError("a paged workload needs the page layout (LayerInputs)")
+                raise ValueError("a paged layout needs page_table, free_pages and pool_pages")
             ps = wl.page_size
             self.page_table = torch.from_numpy(layout.page_table).to(dev)
             self.free_pages = torch.from_numpy(layout.free_pages).to(dev)
             self.out_pt_stride = max((min(b, n) + ps - 1) // ps
                                      for b, n in zip(wl.budgets, wl.lens)) + 1
-            self.desc = desc_from_workload(wl, mode, self.page_table, layout.pool_pages,
+            self.desc = desc_from_spec(wl, mode, self.page_table, layout.pool_pages,
                                            self.out_pt_stride)
             rows = layout.pool_pages * ps
             self.out_page_table = torch.empty((S, self.out_pt_stride), dtype=torch.int32, device=dev)
             self.h_out_page_table = torch.empty(self.out_page_table.shape, dtype=torch.int32).pin_memory()
         else:
-            self.desc = desc_from_workload(wl, mode)
+            self.desc = desc_from_spec(wl, mode)
             rows = self.desc.n_tot
             self.page_table = self.free_pages = self.out_page_table = None
         n_tot, b_tot = self.desc.n_tot, self.desc.b_tot

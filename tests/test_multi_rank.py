@@ -56,3 +56,22 @@ def test_single_rank_needs_no_process_group():
     sharding.barrier(1)
     assert sharding.rank_layers(3, 2) == [300, 301]
     assert abs(sharding.job_throughput(32768, 1, 0.0689) - 32768 / 0.0689e-3) < 1e-3
+
+
+def test_bench_launcher_starts_the_ranks_itself():
+    """`bench.py --gpus 2` without a torchrun environment starts two ranks (here: gloo ranks with
+    a host stub in place of the CUDA step) and rank 0 reports both of them."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items()
+           if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--steps", "3",
+                          "--warmup", "1", "--impl", "stub"], capture_output=True, text=True,
+                         timeout=300, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                      # rank 0 alone prints
+    assert lines[0]["n_gpus"] == 2 and lines[0]["steps"] == 3
+    assert lines[0]["ms_per_step"] >= 2.0 / 3   # the slower rank's time (rank 1 adds 2 ms)
