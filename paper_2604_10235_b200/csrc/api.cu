@@ -211,7 +211,7 @@ int run_fuse(cc_ctx* ctx, const cc_layer_desc* d, const Plan& p, const float* sc
 
 int run_select(cc_ctx* ctx, const cc_layer_desc* d, const Plan& p, const float* fused,
                const float* prior, int32_t* idx, int32_t* count, char* ws, void* stream) {
-  const int cluster = select_cluster_size(p.bt);
+  const int cluster = select_cluster_size(p.bt, p.g.hkv);
   cudaError_t e;
   if (cluster > 0)
     e = launch_select_cluster(make_launch(ctx, stream), p.bt, p.g, d->force_threshold, false,
@@ -422,7 +422,7 @@ int cc_compress_layer(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win,
   float* scores = (float*)(w + p.off_scores);
   float* fused = (float*)(w + p.off_fused);
   if ((rc = run_score(ctx, desc, p, q_win, k, scores, nullptr, w, stream)) != CC_OK) return rc;
-  const int cluster = select_cluster_size(p.bt);
+  const int cluster = select_cluster_size(p.bt, p.g.hkv);
   if (cluster > 0) {
     rc = run_fuse_select(ctx, desc, p, cluster, scores, prior, fused, idx, count, stream);
     if (rc != CC_OK) return rc;

@@ -133,7 +133,7 @@ cudaError_t launch_select(const Launch& L, const BatchTable& bt, const Geometry&
 // cluster kernel: items resident in shared memory, optionally starting from the raw scores
 // (pooling and prior fusion done in the same launch).  select_cluster_size returns the CTAs per
 // (sequence, head) to use, or 0 when a sequence has too many items for it.
-int select_cluster_size(const BatchTable& bt);
+int select_cluster_size(const BatchTable& bt, int hkv);
 cudaError_t launch_select_cluster(const Launch& L, const BatchTable& bt, const Geometry& g,
                                   float force_threshold, bool fused_input, int pool_kind,
                                   int pool_size, float alpha, float beta, const float* scores,

@@ -582,15 +582,28 @@ size_t cluster_smem_bytes(int per, bool fused, int pool_size) {
 }  // namespace
 
 // CTAs per (sequence, head) for the cluster kernel, or 0 when the batch does not fit.
-int select_cluster_size(const BatchTable& bt) {
+// A CTA holds up to kCtaItems items (16 per thread); one CTA of 1024 threads fits per SM, and a
+// cluster is placed inside one GPC, so about 96 CTAs run at a time in clusters of eight, 128 in
+// clusters of four, all 148 otherwise.  Wide clusters finish one (sequence, head) sooner, narrow
+// ones let more of them run at once and pay less per exchange (measured: about 6 + 0.6 x width +
+// items per thread microseconds): the width with the smallest waves x time per wave is taken.
+int select_cluster_size(const BatchTable& bt, int hkv) {
   if (bt.max_items <= 0) return 1;
-  const int target_per = 4;                       // items per thread to aim for
-  int c = 1;
   // in chunk mode a thread reads all tokens of its items, so the width is chosen by tokens
   const long long work = (long long)bt.max_items * bt.chunk;
-  while (c < kMaxCluster && (work + c * kThreads - 1) / (c * kThreads) > target_per) c *= 2;
-  const int per = (bt.max_items + c * kThreads - 1) / (c * kThreads);
-  if (kThreads * per > kCtaItems) return 0;
+  const long long problems = (long long)bt.num_seqs * hkv;
+  auto per_of = [&](int c) { return (bt.max_items + c * kThreads - 1) / (c * kThreads); };
+  auto cost_of = [&](int c) {
+    const long long room = c == 8 ? 96 : (c == 4 ? 128 : 148);
+    const double waves = (double)((problems * c + room - 1) / room);
+    return waves * (6.0 + 0.6 * c + 1.05 * (double)((work + c * kThreads - 1) / (c * kThreads)));
+  };
+  // widest useful cluster: four items per thread ...
+  int c = 1;
+  while (c < kMaxCluster && (work + c * kThreads - 1) / (c * kThreads) > 4) c *= 2;
+  if (kThreads * per_of(c) > kCtaItems) return 0;
+  // ... narrowed while the batch needs several waves and fewer, longer waves are cheaper
+  while (c > 1 && kThreads * per_of(c / 2) <= kCtaItems && cost_of(c / 2) < cost_of(c)) c /= 2;
   return c;
 }
 
