@@ -47,7 +47,10 @@ SM_COUNT = 148
 # DRAM bytes (read + write) of the two launches of the score stage, per workload, from the ncu
 # captures summarised under profiles/ (counters taken on the kernel as it stands in this tree):
 # "live" = caches left alone between the launches, "flushed" = ncu's default cache flush.
-SCORE_TRAFFIC_BYTES = {}
+SCORE_TRAFFIC_BYTES = {
+    "llama3_8b": {"live": 72.9e6, "flushed": 136.2e6},          # algorithmic: 68.2 MB
+    "ragged_paged": {"live": 1210.5e6, "flushed": 1219.9e6},    # algorithmic: 614.1 MB
+}
 
 
 def load_peaks():

@@ -123,6 +123,15 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       "[%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+// K tile copy with an L2 eviction-priority hint: pass 1 asks L2 to keep the tile (pass 2 reads
+// it again), pass 2 marks it as the first to go.
+__device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                                 int c0, int c1, int c2, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4, %5}], [%2], %6;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
                                             int c0, int c1, int c2, int c3) {
   asm volatile(
@@ -456,6 +465,9 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
       int stage = 0, cur_problem = -1;
       uint32_t phase = 0, qe_phase = 0;
       const int ps = bt.page_size;
+      uint64_t k_policy;
+      if (PASS == 1) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(k_policy));
+      else           asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(k_policy));
       for (int t = t_begin; t < t_end; ++t, cur.advance(bt, g.hkv)) {
         const SeqInfo& sq = bt.seq[cur.s];
         if (cur.problem(g.hkv) != cur_problem) {
@@ -489,8 +501,8 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
         if (ps == 0) {
           if (lane == 0) {
             mbar_expect_tx(fb, kStageBytes);
-            tma_load_3d(dst, &k_map, fb, 0, cur.h, sq.tok_off + key0);
-            tma_load_3d(dst + kPanelBytes, &k_map, fb, 64, cur.h, sq.tok_off + key0);
+            tma_load_3d_hint(dst, &k_map, fb, 0, cur.h, sq.tok_off + key0, k_policy);
+            tma_load_3d_hint(dst + kPanelBytes, &k_map, fb, 64, cur.h, sq.tok_off + key0, k_policy);
           }
         } else {
           const bool good = mine && page_id >= 0 && ((int64_t)page_id + 1) * ps <= P.pool_rows;
@@ -502,8 +514,8 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
           __syncwarp();
           if (good) {
             const uint32_t off = (uint32_t)lane * (uint32_t)ps * 128u;
-            tma_load_3d(dst + off, &k_map, fb, 0, cur.h, page_id * ps);
-            tma_load_3d(dst + kPanelBytes + off, &k_map, fb, 64, cur.h, page_id * ps);
+            tma_load_3d_hint(dst + off, &k_map, fb, 0, cur.h, page_id * ps, k_policy);
+            tma_load_3d_hint(dst + kPanelBytes + off, &k_map, fb, 64, cur.h, page_id * ps, k_policy);
           }
         }
         if (++stage == P.n_stages) { stage = 0; phase ^= 1; }
