@@ -36,12 +36,11 @@ UNIT = "tokens/s/layer"
 L2_BYTES = 126e6
 TIMED_BLOCKS = 50         # the block of --steps steps is timed this many times; the median counts
 
-# Exponentials per clock per SM of the score kernel's inner loop (special-function unit plus the
-# packed-FMA polynomial, 7 pairs in 16 on the FMA pipe), measured on a B200 with the loop alone on
-# 16 warps per SM: values held in registers / values read from tensor memory as the kernel does.
-# Source: profiles/exp_throughput_microbenchmark.md.
-EXP_PER_CLK_SM_REGISTERS = 22.6
-EXP_PER_CLK_SM_TMEM = 17.6
+# Exponentials per clock per SM of the score kernel's inner loop run alone on 16 warps per SM
+# (special-function unit plus the packed-FMA polynomial): values held in registers / values read
+# from tensor memory as the kernel does.  Measured at start-up through cc_exp_rate_probe; these
+# are the figures of an earlier run, used only if the probe is not run.
+EXP_RATE = {"registers": 22.0, "tmem": 17.5, "source": "earlier run"}
 SM_COUNT = 148
 
 # DRAM bytes (read + write) of the two launches of the score stage, per workload, from the ncu
@@ -95,9 +94,9 @@ def roofline_of(work, peaks, seconds, clock_mhz=None):
            "frac": t_roof / seconds}
     if clock_mhz:
         # both passes of the score stage evaluate every exponential once
-        per_s = EXP_PER_CLK_SM_REGISTERS * SM_COUNT * clock_mhz * 1e6
+        per_s = EXP_RATE["registers"] * SM_COUNT * clock_mhz * 1e6
         out["exp_bound_us"] = 2.0 * work["exps"] / per_s * 1e6
-        out["exp_bound_us_tmem_reads"] = 2.0 * work["exps"] / (EXP_PER_CLK_SM_TMEM * SM_COUNT * clock_mhz * 1e6) * 1e6
+        out["exp_bound_us_tmem_reads"] = 2.0 * work["exps"] / (EXP_RATE["tmem"] * SM_COUNT * clock_mhz * 1e6) * 1e6
     return out
 
 
@@ -389,6 +388,8 @@ def run_ours(args, wl):
     ctx = cc.Context(local)
     peaks = load_peaks()
     work = algorithmic_work(wl)
+    EXP_RATE.update(registers=cc.cc_exp_rate_probe(ctx, False), tmem=cc.cc_exp_rate_probe(ctx, True),
+                    source="cc_exp_rate_probe, this run")
 
     # inputs: layer sets resident in HBM before timing, plus pinned host copies of two of them
     run = WorkloadRun(ctx, wl, rank, pinned=True)
@@ -493,6 +494,7 @@ def run_ours(args, wl):
         path = roofline_of(work, peaks, ms_step * 1e-3, clock_mhz)
         path.update({"bytes": work["bytes"], "flops": work["flops"], "exps_per_pass": work["exps"],
                      "hbm_peak_gbs": peaks["hbm_gbs"], "tensor_peak_tflops": peaks["bf16_tflops"],
+                     "exp_per_clk_per_sm": dict(EXP_RATE),
                      "binding_unit": "special-function unit + FMA pipe + instruction issue of the "
                                      "exponentials (see exp_bound_us), not HBM or the tensor pipe"})
         line = {

@@ -114,7 +114,7 @@ typedef struct cc_layer_desc {
 } cc_layer_desc;
 
 /* Creates a context on CUDA device `device` (must be compute capability 10.x).  Allocates a
- * few hundred bytes of device and pinned host memory for the status word; the only
+ * few KB of device and pinned host memory (status word, scratch of the probe); the only
  * allocation the library ever makes.  *out is untouched on failure. */
 int cc_create(cc_ctx** out, int device);
 /* Frees the context.  The caller must have synchronised every stream that used it. */
@@ -260,6 +260,17 @@ int cc_select_spans(const int32_t* starts, const int32_t* ends, const float* sco
                     const uint8_t* is_protected, int32_t num_spans, int32_t n, int32_t budget,
                     double span_ratio, int32_t span_min, float* prior_mask, int32_t* taken,
                     int32_t* num_taken);
+
+/* (No counterpart in the paper: a measurement aid.)  Throughput of the inner loop that bounds
+ * cc_score_window - acc += 2^(v * c + off), two pairs of values in three on the special-function
+ * unit and one on the FMA pipe - with sixteen warps per SM doing nothing else for `iters` rounds of
+ * 32 values per thread: values held in registers (from_tmem == 0) or read from tensor memory the
+ * way the kernel reads its accumulators (from_tmem != 0).  *per_clock_per_sm (HOST) receives the
+ * mean over the SMs of values per SM clock.  Multiplied by the SM count and the SM clock it is
+ * the exponential ceiling of the score stage, which evaluates 2 * w * G exponentials per (key,
+ * KV head).  Uses a few KB of device memory owned by the context; synchronises `stream`. */
+int cc_exp_rate_probe(cc_ctx* ctx, int32_t from_tmem, int32_t iters, double* per_clock_per_sm,
+                      void* stream);
 
 /* Device pointers, inside the workspace last given to cc_compress_layer for `desc`, of the
  * intermediate scores [H_kv][N_tot] and fused values [H_kv][M_tot] (for inspection). */

@@ -31,7 +31,7 @@ EXPORTS = ("cc_create", "cc_destroy", "cc_status_string", "cc_last_error", "cc_p
            "cc_workspace_bytes", "cc_score_window", "cc_fuse_prior_pool", "cc_topk_select",
            "cc_compact_kv", "cc_compress_layer", "cc_workspace_views", "cc_topk_select_static",
            "cc_structural_score", "cc_plan_budgets", "cc_select_spans", "cc_ppl_chunk_scores",
-           "cc_select_chunks")
+           "cc_select_chunks", "cc_exp_rate_probe")
 CC_STATIC_SELECT_MAX_ITEMS = 1 << 20
 
 
@@ -102,6 +102,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.cc_select_spans.argtypes = [vp, vp, vp, vp, C.c_int32, C.c_int32, C.c_int32, C.c_double,
                                     C.c_int32, vp, vp, vp]
     lib.cc_compress_layer.argtypes = [vp, dp] + [vp] * 10 + [vp, sz, vp]
+    lib.cc_exp_rate_probe.argtypes = [vp, C.c_int32, C.c_int32, C.POINTER(C.c_double), vp]
     lib.cc_workspace_views.argtypes = [vp, dp, vp, C.POINTER(vp), C.POINTER(vp)]
     for name in EXPORTS:
         if name not in ("cc_status_string", "cc_last_error", "cc_workspace_bytes"):
@@ -354,6 +355,14 @@ def cc_compress_layer(ctx: Context, desc: Desc, q_win, k, v, prior, k_out, v_out
                                         _ptr(prior), _ptr(k_out), _ptr(v_out), _ptr(idx),
                                         _ptr(count), _ptr(free_pages), _ptr(out_page_table),
                                         _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def cc_exp_rate_probe(ctx: Context, from_tmem: bool, iters: int = 4000, stream=None) -> float:
+    """Values per clock per SM of the score kernel's inner loop run alone (synchronises)."""
+    rate = C.c_double(0.0)
+    ctx.check(ctx.lib.cc_exp_rate_probe(ctx.handle, 1 if from_tmem else 0, iters, C.byref(rate),
+                                        _stream(stream)))
+    return float(rate.value)
 
 
 def cc_workspace_views(ctx: Context, desc: Desc, ws: torch.Tensor):

@@ -12,7 +12,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB_DIR = os.path.join(HERE, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "libcodecomp.so")
 SOURCES = ["api.cu", "score_simt.cu", "score_tc.cu", "fuse_pool.cu", "select.cu", "select_cluster.cu", "compact.cu",
-           "str_score.cu", "planner.cu", "ppl.cu"]
+           "str_score.cu", "planner.cu", "ppl.cu", "exp_probe.cu"]
 
 
 def nvcc_path() -> str:

@@ -13,6 +13,7 @@ struct cc_ctx {
   int sm_count;
   cc::DeviceStatus* d_status;
   cc::DeviceStatus* h_status;   // pinned
+  long long* d_probe;           // scratch of cc_exp_rate_probe: two words per SM
   void* encode_tiled;           // cuTensorMapEncodeTiled, resolved through the runtime
   char err[256];
 };
@@ -277,6 +278,7 @@ int cc_create(cc_ctx** out, int device) {
   ctx->sm_count = prop.multiProcessorCount;
   bool ok = cudaMalloc(&ctx->d_status, sizeof(cc::DeviceStatus)) == cudaSuccess &&
             cudaMemset(ctx->d_status, 0, sizeof(cc::DeviceStatus)) == cudaSuccess &&
+            cudaMalloc(&ctx->d_probe, 2 * 256 * sizeof(long long)) == cudaSuccess &&
             cudaMallocHost(&ctx->h_status, sizeof(cc::DeviceStatus)) == cudaSuccess;
   if (ok) {
     cudaDriverEntryPointQueryResult qres;
@@ -287,6 +289,7 @@ int cc_create(cc_ctx** out, int device) {
   cudaSetDevice(prev);
   if (!ok) {
     if (ctx->d_status) cudaFree(ctx->d_status);
+    if (ctx->d_probe) cudaFree(ctx->d_probe);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
     delete ctx;
     return CC_ERR_CUDA;
@@ -298,6 +301,7 @@ int cc_create(cc_ctx** out, int device) {
 int cc_destroy(cc_ctx* ctx) {
   if (!ctx) return CC_ERR_INVALID_ARG;
   cudaFree(ctx->d_status);
+  cudaFree(ctx->d_probe);
   cudaFreeHost(ctx->h_status);
   delete ctx;
   return CC_OK;
@@ -487,6 +491,16 @@ int cc_select_chunks(cc_ctx* ctx, const float* score, int32_t num_chunks, int32_
   if (!score || !chosen) return fail(ctx, CC_ERR_INVALID_ARG, "NULL tensor pointer");
   cudaError_t e = launch_select_chunks(make_launch(ctx, stream), score, num_chunks, k, chosen);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "chunk selection launch");
+  return CC_OK;
+}
+
+int cc_exp_rate_probe(cc_ctx* ctx, int32_t from_tmem, int32_t iters, double* per_clock_per_sm,
+                      void* stream) {
+  if (!ctx || !per_clock_per_sm) return CC_ERR_INVALID_ARG;
+  if (iters < 1 || iters > (1 << 24)) return fail(ctx, CC_ERR_INVALID_ARG, "iters must be in [1, 2^24]");
+  cudaError_t e = run_exp_probe(make_launch(ctx, stream), from_tmem != 0, iters, ctx->d_probe,
+                                per_clock_per_sm);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "exponential-rate probe");
   return CC_OK;
 }
 

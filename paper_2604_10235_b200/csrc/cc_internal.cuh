@@ -162,4 +162,8 @@ cudaError_t launch_str_score(const Launch& L, const BatchTable& bt, const Geomet
                              float threshold, const int32_t* idx, const float* prior,
                              float* score, int32_t* counts);
 
+// throughput probe of the score kernel's inner loop (exp_probe.cu)
+cudaError_t run_exp_probe(const Launch& L, bool from_tmem, int iters, long long* scratch,
+                          double* rate);
+
 }  // namespace cc

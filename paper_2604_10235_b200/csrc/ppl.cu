@@ -12,6 +12,7 @@
 #include <math.h>
 
 #include "cc_internal.cuh"
+#include "exp2_poly.cuh"
 
 namespace cc {
 
@@ -20,24 +21,6 @@ namespace {
 constexpr int kThreads = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-
-__device__ __forceinline__ float ex2f(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-// 2^x on the FMA pipe for x <= 0: round to the nearest integer through the 1.5 * 2^23 trick,
-// degree-3 minimax polynomial for the fraction in [-0.5, 0.5] (relative error 7.8e-5), integer
-// part added into the exponent field; arguments below -125 are clamped (their value is ~0).
-__device__ __forceinline__ float ex2_poly(float x) {
-  x = fmaxf(x, -125.0f);
-  const float t = x + 12582912.0f;
-  const float f = x - (t - 12582912.0f);
-  float p = fmaf(f, 0.05516434833407402f, 0.24259322881698608f);
-  p = fmaf(p, f, 0.693260669708252f);
-  p = fmaf(p, f, 0.9999293088912964f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
-}
 
 __device__ __forceinline__ float max3f(float a, float b, float c) {
   float d;
@@ -51,23 +34,23 @@ struct Running {
   __device__ __forceinline__ void add8(const float (&x)[8]) {
     const float vm = max3f(max3f(x[0], x[1], x[2]), max3f(x[3], x[4], x[5]), fmaxf(x[6], x[7])) * kLog2e;
     if (vm > m) {
-      s *= ex2f(m - vm);          // m = -inf at the start: the factor is 0 and s is 0
+      s *= ex2(m - vm);          // m = -inf at the start: the factor is 0 and s is 0
       m = vm;
     }
     const float nm = -m;
     float a = 0.f, b = 0.f;
 #pragma unroll
     for (int i = 0; i < 8; i += 2) {
-      a += ex2f(fmaf(x[i], kLog2e, nm));
+      a += ex2(fmaf(x[i], kLog2e, nm));
       // one value in eight goes to the FMA pipe, which otherwise idles
-      b += (i == 2) ? ex2_poly(fmaf(x[i + 1], kLog2e, nm)) : ex2f(fmaf(x[i + 1], kLog2e, nm));
+      b += (i == 2) ? ex2_poly(fmaf(x[i + 1], kLog2e, nm)) : ex2(fmaf(x[i + 1], kLog2e, nm));
     }
     s += a + b;
   }
   __device__ __forceinline__ void merge(float om, float os) {
     const float nm = fmaxf(m, om);
     if (nm == -INFINITY) return;
-    s = s * ex2f(m - nm) + os * ex2f(om - nm);
+    s = s * ex2(m - nm) + os * ex2(om - nm);
     m = nm;
   }
 };

@@ -385,3 +385,13 @@ def test_structural_score_of_the_fused_path_on_tiny():
                                 wl.budget, wl.alpha, wl.beta, wl.force_threshold)
     for h in range(hkv):
         assert orc.structural_score(res["idx"][h], x.prior, wl.force_threshold)[0] == 1.0
+
+
+def test_exp_rate_probe_reports_a_plausible_rate():
+    """Between the special-function unit alone (16 per clock per SM, minus the share that the
+    polynomial takes over) and what both pipes could do if nothing else limited them."""
+    reg = cc.cc_exp_rate_probe(ctx(), False, 2000)
+    tm = cc.cc_exp_rate_probe(ctx(), True, 2000)
+    assert 12.0 < reg < 40.0, reg
+    assert 8.0 < tm < 40.0, tm
+    assert ctx().poll() == 0
