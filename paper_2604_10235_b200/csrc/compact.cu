@@ -23,7 +23,7 @@ __device__ __forceinline__ void st_stream(uint4* p, uint4 v) {
 }
 
 // grid: (blocks over slot*head pairs of the longest sequence, num_seqs)
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 8)      // 32 registers: eight blocks, all warp slots of an SM
 compact_kernel(const __grid_constant__ BatchTable bt, const Geometry g,
                const uint16_t* __restrict__ k, const uint16_t* __restrict__ v,
                const int32_t* __restrict__ idx, uint16_t* __restrict__ k_out,
