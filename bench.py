@@ -614,6 +614,11 @@ def main():
         return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     from paper_2604_10235_b200 import inputs as gen
+    if args.workload == "chunk_scoring":
+        # the chunk-selection kernel alone (Section 4.1; not part of a compression step)
+        from paper_2604_10235_b200 import binding as cc
+        print(json.dumps({"chunk_scoring": chunk_scoring_bandwidth(cc.Context(0), load_peaks())}), flush=True)
+        return
     wl = {**gen.workloads(), **bench_workloads()}[args.workload]
     if args.impl == "reference":
         run_reference(args, wl)

@@ -1,8 +1,8 @@
 /*
  * codecomp.h - C ABI of the CodeComp per-layer KV-cache compression step on one B200.
  *
- * The step runs once per transformer layer after prefill (paper, Section 4.5:
- * "Compression is applied independently at each transformer layer"):
+ * The step runs once per transformer layer after prefill; every layer is compressed on its own
+ * (Section 4.5):
  *
  *   score   u_h(j) = sum over the window rows t and the query heads g of KV head h of
  *           softmax_j( q_{g,t} . k_j / sqrt(d) )                       (Section 4.5)
@@ -192,8 +192,9 @@ int cc_compress_layer(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win,
                       int32_t* idx, int32_t* count, const int32_t* free_pages,
                       int32_t* out_page_table, void* ws, size_t ws_bytes, void* stream);
 
-/* Str. Score (Section 5.3, caption of the bug-localization table: "the average fraction of
- * structurally critical tokens retained across layers and chunks").  For every sequence s and
+/* Str. Score (Section 5.3, caption of the bug-localization table): the share of the structurally
+ * critical tokens that survives compression, which the paper averages over layers and chunks.
+ * For every sequence s and
  * KV head h: score[s][h] = |{i : prior[idx[h][i]] >= threshold}| / |{j : prior[j] >= threshold}|,
  * 1 when the sequence has no such token; the average over layers and chunks is the caller's.
  * idx: device i32 [H_kv][B_tot] as written by cc_topk_select / cc_compress_layer (entries < 0

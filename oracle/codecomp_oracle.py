@@ -45,7 +45,8 @@ unpinned" by the paper, pinned here only by self-consistency tests):
   - the edge rule of average pooling (zero padding, always divide by the width);
   - the ``causal`` option of ``window_scores`` (window inside the sequence) is an extension;
     the paper's window follows the context and needs no mask;
-  - ``select_spans``: "added greedily until the span budget is exhausted" is read as: spans
+  - ``select_spans``: the greedy filling of the span budget (Section 4.4, "Span selection
+    under budget") is read as: spans
     are taken whole, in rank order (score descending, earlier start first), while the
     tokens covered so far are fewer than B^span, so the last span taken may overshoot it;
   - ``structural_score`` of a sequence without structurally critical tokens is taken

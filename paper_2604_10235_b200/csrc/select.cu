@@ -11,6 +11,7 @@
 // final ordered pass resolves ties towards lower indices with one block-wide prefix sum and
 // writes ascending token indices.
 #include "cc_internal.cuh"
+#include "select_common.cuh"
 
 namespace cc {
 
@@ -29,16 +30,7 @@ struct Shared {
   unsigned bcast[4];
 };
 
-__device__ __forceinline__ unsigned mono_key(float x) {
-  unsigned b = __float_as_uint(__fadd_rn(x, 0.0f));
-  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-}
 
-__device__ __forceinline__ unsigned warp_sum(unsigned v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
 
 __device__ unsigned block_sum(Shared& sm, unsigned v) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;

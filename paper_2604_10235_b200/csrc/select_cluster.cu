@@ -20,6 +20,7 @@
 #include <string.h>
 
 #include "cc_internal.cuh"
+#include "select_common.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -59,17 +60,8 @@ struct ClusterParams {
   int32_t* count;
 };
 
-__device__ __forceinline__ unsigned mono_key(float x) {
-  unsigned b = __float_as_uint(__fadd_rn(x, 0.0f));
-  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-}
 __host__ __device__ __forceinline__ int padded(int li) { return li + (li >> 5); }
 
-__device__ __forceinline__ unsigned warp_sum(unsigned v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
 
 struct Ctx {
   Shared* sm;

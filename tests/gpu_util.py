@@ -57,6 +57,14 @@ def assert_scores_close(u: np.ndarray, u_ref: np.ndarray, rows: int, n: int, tol
     bad = err > bound
     assert not bad.any(), (f"{bad.sum()} of {bad.size} scores off; worst ratio "
                            f"{(err / bound).max():.3g} at {np.unravel_index((err / bound).argmax(), err.shape)}")
+    # The floor above (one mean score) only matters for scores far below the mean.  Every score
+    # that is not negligible (above a thousandth of the mean) must also meet the relative bound
+    # with hardly any help from the floor: the kernels' error sources are relative.
+    mean = rows / max(n, 1)
+    sizable = np.abs(u_ref) > 1e-3 * mean
+    rel_bad = sizable & (err > tol * np.abs(u_ref) + tol * 1e-3 * mean)
+    assert not rel_bad.any(), (f"{rel_bad.sum()} of {sizable.sum()} sizable scores miss the relative "
+                               f"bound; worst {(err[sizable] / np.abs(u_ref[sizable])).max():.3g}")
 
 
 def seq_kv(x: gen.LayerInputs, s: int):
