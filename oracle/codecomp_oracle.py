@@ -18,6 +18,9 @@ What each function follows:
 * ``fuse_prior``      - Section 4.4 "Span scoring" (importance is a weighted sum of
                         structural indicators and an attention term, Appendix
                         "Structural prior configuration").
+* ``nearest_fill_values`` - Section 4.4 "Token-level protection", last sentence: when the
+                        protected tokens do not fill the budget, the rest goes to the tokens
+                        nearest to them (the alternative to the attention fill of Section 4.5).
 * ``chunk_reduce``    - chunk-level aggregation of scores and prior (benchmark variant).
 * ``span_budget``     - Section 4.4, the equation for B^span.
 * ``select_tokens``   - Section 4.4 "Token-level protection" (protected tokens first,
@@ -50,7 +53,10 @@ unpinned" by the paper, pinned here only by self-consistency tests):
     are taken whole, in rank order (score descending, earlier start first), while the
     tokens covered so far are fewer than B^span, so the last span taken may overshoot it;
   - ``structural_score`` of a sequence without structurally critical tokens is taken
-    as 1 (nothing could be lost); the paper does not say.
+    as 1 (nothing could be lost); the paper does not say;
+  - ``nearest_fill_values``: "nearest" is the distance in token positions to the closest token
+    whose prior reaches the threshold (before any cap of the protected set), equal distances go
+    to the lower index, and a sequence without such a token keeps its first tokens.
 """
 from __future__ import annotations
 
@@ -141,6 +147,31 @@ def fuse_prior(pooled: np.ndarray, prior: np.ndarray, alpha: float, beta: float,
     t1 = (a * np.asarray(pooled, dtype=dtype)).astype(dtype)
     t2 = (b * np.asarray(prior, dtype=dtype)).astype(dtype)
     return (t1 + t2).astype(dtype)
+
+
+def nearest_fill_values(prior: np.ndarray, force_threshold: float) -> np.ndarray:
+    """Ranking value of every token when the budget left by the protected tokens is filled with
+    the tokens nearest to them: minus the distance (in positions) to the closest token with
+    prior >= force_threshold, found with one forward and one backward sweep.  Larger is better,
+    so the usual order (value descending, index ascending) takes nearer tokens first and the
+    lower index among equally near ones.  Without any such token every value is minus the
+    sequence length (the order is then by index)."""
+    n = len(prior)
+    hit = np.asarray(prior).astype(np.float32) >= np.float32(force_threshold)
+    dist = np.full(n, n, dtype=np.int64)
+    last = -1
+    for j in range(n):                         # distance to the closest protected token at or before j
+        if hit[j]:
+            last = j
+        if last >= 0:
+            dist[j] = j - last
+    nxt = -1
+    for j in range(n - 1, -1, -1):             # ... and at or after j
+        if hit[j]:
+            nxt = j
+        if nxt >= 0:
+            dist[j] = min(dist[j], nxt - j)
+    return -dist.astype(np.float64)
 
 
 # --------------------------------------------------------------------------- A6 chunks
@@ -364,7 +395,8 @@ def compress_sequence(q_bits: np.ndarray, k_bits: np.ndarray, v_bits: Optional[n
                       prior: np.ndarray, n_heads_kv: int, pool_kind: int, pool_size: int,
                       budget: int, alpha: float, beta: float, force_threshold: float,
                       span_ratio: float = 0.0, span_min: int = 0, chunk: int = 1,
-                      stage_dtype=np.float64, causal: bool = False) -> dict:
+                      stage_dtype=np.float64, causal: bool = False,
+                      nearest_fill: bool = False) -> dict:
     """The whole per-layer step for one contiguous sequence.
 
     q_bits [w][H_q][d], k_bits/v_bits [n][H_kv][d] as bf16 bit patterns, prior [n].
@@ -384,6 +416,11 @@ def compress_sequence(q_bits: np.ndarray, k_bits: np.ndarray, v_bits: Optional[n
         pooled = pool_scores(u_s, pool_kind, pool_size, dtype=stage_dtype)
         item_p = prior_s
     fused = fuse_prior(pooled, item_p[None, :], alpha, beta, dtype=stage_dtype)
+    if nearest_fill:
+        # Section 4.4 fill rule instead of the attention scores (token level only)
+        assert chunk == 1
+        fused = np.repeat(nearest_fill_values(prior, force_threshold)[None, :], n_heads_kv, axis=0
+                          ).astype(stage_dtype)
     idx = [select_tokens(fused[h], item_p, n, budget, force_threshold, span_ratio,
                          span_min, chunk) for h in range(n_heads_kv)]
     res = {"scores": u, "lse": lse, "pooled": pooled, "fused": fused, "idx": idx,

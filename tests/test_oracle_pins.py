@@ -612,3 +612,38 @@ def test_select_chunks_lowest_first_with_ties():
     got = orc.select_chunks(r, 10)
     assert np.array_equal(np.sort(r)[:10], r[got])           # against the library sort
     assert all(r[a] < r[b] or (r[a] == r[b] and a < b) for a, b in zip(got[:-1], got[1:]))
+
+
+# ------------------------------------------------------------------ nearest-to-protected fill
+def test_nearest_fill_hand_cases():
+    """Section 4.4, last sentence of "Token-level protection": worked by hand."""
+    #            0  1  2  3  4  5  6  7  8  9
+    prior = np.array([0, 0, 1, 0, 0, 0, 0, 1, 0, 0], np.float32)
+    assert (-orc.nearest_fill_values(prior, 0.5)).tolist() == [2, 1, 0, 1, 2, 2, 1, 0, 1, 2]
+    # budget 6: the two protected tokens, then distance 1 (1, 3, 6, 8 in index order)
+    assert orc.select_tokens(orc.nearest_fill_values(prior, 0.5), prior, 10, 6, 0.5).tolist() == [1, 2, 3, 6, 7, 8]
+    # budget 5: of the four tokens at distance 1 the three with the lowest index
+    assert orc.select_tokens(orc.nearest_fill_values(prior, 0.5), prior, 10, 5, 0.5).tolist() == [1, 2, 3, 6, 7]
+    # no protected token: the first tokens of the sequence
+    none = np.zeros(7, np.float32)
+    assert (-orc.nearest_fill_values(none, 0.5)).tolist() == [7] * 7
+    assert orc.select_tokens(orc.nearest_fill_values(none, 0.5), none, 7, 3, 0.5).tolist() == [0, 1, 2]
+    # protected token at one end only
+    end = np.array([0, 0, 0, 0, 1], np.float32)
+    assert (-orc.nearest_fill_values(end, 0.5)).tolist() == [4, 3, 2, 1, 0]
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_nearest_fill_vs_quadratic_loop(seed):
+    rng = np.random.Generator(np.random.PCG64(900 + seed))
+    n = int(rng.integers(1, 120))
+    prior = (rng.random(n) < rng.choice([0.0, 0.05, 0.3])).astype(np.float32) * np.float32(0.8)
+    got = -orc.nearest_fill_values(prior, 0.5)
+    prot = [j for j in range(n) if prior[j] >= 0.5]
+    want = [min((abs(j - p) for p in prot), default=n) for j in range(n)]
+    assert got.tolist() == want
+    # the retained set: every protected token, then by (distance, index)
+    b = int(rng.integers(0, n + 1))
+    ref = sorted(sorted(range(n), key=lambda j: (0 if prior[j] >= 0.5 else 1, want[j], j))[:b]) \
+        if len(prot) <= b else prot[:b]
+    assert orc.select_tokens(-got, prior, n, b, 0.5).tolist() == ref
