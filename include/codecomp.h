@@ -74,6 +74,9 @@ extern "C" {
 #define CC_POOL_MAX    1
 #define CC_POOL_AVG    2
 #define CC_MAX_SEQS    64
+#define CC_FILL_ATTENTION 0 /* budget left by the protected tokens: top-ranked fused scores (Section 4.5) */
+#define CC_FILL_NEAREST   1 /* ... or the tokens nearest to a protected token (Section 4.4, last sentence of
+                               "Token-level protection") */
 
 typedef struct cc_ctx cc_ctx;
 
@@ -111,6 +114,12 @@ typedef struct cc_layer_desc {
                                window is the last w tokens of the sequence itself; row t sits at
                                position n_s - w + t and attends to keys j <= n_s - w + t only.
                                Needs n_s >= w for every non-empty sequence. */
+  int32_t fill_mode;        /* CC_FILL_ATTENTION (default) or CC_FILL_NEAREST: the value that ranks the
+                               unprotected tokens is minus the distance, in token positions, to the
+                               closest token with prior >= force_threshold (equal distances: lower
+                               index first; no such token: the first tokens of the sequence).  The
+                               attention scores then play no part in the selection and
+                               cc_compress_layer does not compute them.  Token level only. */
 } cc_layer_desc;
 
 /* Creates a context on CUDA device `device` (must be compute capability 10.x).  Allocates a
@@ -141,7 +150,8 @@ int cc_score_window(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win, c
 /* A2+A3 - pooling (Appendix "Compression settings") and prior fusion (Section 4.4 "Span
  * scoring").  Token level: fused[h][j] = alpha * pool(scores[h])[j] + beta * prior[j], every
  * operation rounded to f32, average pooling = left-to-right sum of the k zero-padded taps
- * divided by k, max pooling over the valid taps.  Chunk level (chunk_size > 1): the item
+ * divided by k, max pooling over the valid taps.  With fill_mode == CC_FILL_NEAREST the value is
+ * minus the distance to the closest protected token instead (scores may be NULL).  Chunk level (chunk_size > 1): the item
  * value is the in-order f32 sum of the chunk's scores and the prior is the chunk's maximum.
  * scores, prior, fused: device f32.  Needs no workspace. */
 int cc_fuse_prior_pool(cc_ctx* ctx, const cc_layer_desc* desc, const float* scores,

@@ -39,6 +39,7 @@ class LayerSpec:
     span_min: int = 0
     page_size: int = 0                    # 0 = contiguous K/V
     causal: bool = False
+    fill_mode: int = cc.CC_FILL_ATTENTION
 
     @classmethod
     def like(cls, obj) -> "LayerSpec":
@@ -60,7 +61,7 @@ def desc_from_spec(wl: LayerSpec, mode: int = cc.CC_MODE_BF16,
               pool_size=wl.pool_size, chunk_size=wl.chunk_size, alpha=wl.alpha, beta=wl.beta,
               force_threshold=wl.force_threshold, span_ratio=wl.span_ratio, span_min=wl.span_min,
               page_size=wl.page_size, page_table=page_table, pool_pages=pool_pages,
-              out_page_table_stride=out_pt_stride, causal=wl.causal)
+              out_page_table_stride=out_pt_stride, causal=wl.causal, fill_mode=wl.fill_mode)
     if len(wl.lens) > 1 or wl.page_size:
         return cc.Desc(wl.n_heads_q, wl.n_heads_kv, wl.window, seq_lens=wl.lens,
                        budgets=wl.budgets, **kw)

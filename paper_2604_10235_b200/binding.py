@@ -26,6 +26,7 @@ CC_F32 = 2
 CC_MODE_BF16, CC_MODE_FP32 = 0, 1
 CC_POOL_NONE, CC_POOL_MAX, CC_POOL_AVG = 0, 1, 2
 CC_MAX_SEQS = 64
+CC_FILL_ATTENTION, CC_FILL_NEAREST = 0, 1
 
 EXPORTS = ("cc_create", "cc_destroy", "cc_status_string", "cc_last_error", "cc_poll_status",
            "cc_workspace_bytes", "cc_score_window", "cc_fuse_prior_pool", "cc_topk_select",
@@ -57,7 +58,7 @@ class cc_layer_desc(C.Structure):
         ("page_table", C.c_void_p),
         ("page_table_stride", C.c_int32), ("pool_pages", C.c_int32),
         ("out_page_table_stride", C.c_int32),
-        ("causal", C.c_int32),
+        ("causal", C.c_int32), ("fill_mode", C.c_int32),
     ]
 
 
@@ -175,7 +176,8 @@ class Desc:
                  pool_size: int = 7, chunk_size: int = 1, alpha: float = 1.0, beta: float = 0.0,
                  force_threshold: float = math.inf, span_ratio: float = 0.0, span_min: int = 0,
                  page_size: int = 0, page_table: Optional[torch.Tensor] = None, pool_pages: int = 0,
-                 out_page_table_stride: int = 0, causal: bool = False, q_strides=None,
+                 out_page_table_stride: int = 0, causal: bool = False, fill_mode: int = 0,
+                 q_strides=None,
                  kv_strides=None,
                  out_strides=(0, 0)):
         c = cc_layer_desc()
@@ -210,6 +212,7 @@ class Desc:
         c.pool_pages = pool_pages
         c.out_page_table_stride = out_page_table_stride
         c.causal = 1 if causal else 0
+        c.fill_mode = fill_mode
         self.c = c
 
     # sizes the caller needs to allocate outputs

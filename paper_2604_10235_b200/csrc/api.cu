@@ -77,6 +77,10 @@ int build_plan(cc_ctx* ctx, const cc_layer_desc* d, Plan* p) {
     return fail(ctx, CC_ERR_UNSUPPORTED, "pool_size must be odd and at most 63");
   if (d->chunk_size > 1 && d->pool_kind != CC_POOL_NONE && d->pool_size > 1)
     return fail(ctx, CC_ERR_UNSUPPORTED, "chunk-level ranking takes no pooling");
+  if (d->fill_mode != CC_FILL_ATTENTION && d->fill_mode != CC_FILL_NEAREST)
+    return fail(ctx, CC_ERR_INVALID_ARG, "unknown fill_mode");
+  if (d->fill_mode == CC_FILL_NEAREST && d->chunk_size > 1)
+    return fail(ctx, CC_ERR_UNSUPPORTED, "the nearest-token fill is token level only");
   if (isnan(d->alpha) || isnan(d->beta) || isnan(d->force_threshold))
     return fail(ctx, CC_ERR_INVALID_ARG, "alpha, beta and force_threshold must not be NaN");
   if (d->num_seqs < 0 || d->num_seqs > CC_MAX_SEQS)
@@ -204,6 +208,11 @@ int run_score(cc_ctx* ctx, const cc_layer_desc* d, const Plan& p, const void* q,
 int run_fuse(cc_ctx* ctx, const cc_layer_desc* d, const Plan& p, const float* scores,
              const float* prior, float* fused, void* stream) {
   if (p.bt.m_tot == 0) return CC_OK;
+  if (d->fill_mode == CC_FILL_NEAREST) {
+    cudaError_t e = launch_nearest_fill(make_launch(ctx, stream), p.bt, p.g, d->force_threshold, prior, fused);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "nearest-fill launch");
+    return CC_OK;
+  }
   cudaError_t e = launch_fuse_pool(make_launch(ctx, stream), p.bt, p.g, d->pool_kind, d->pool_size,
                                    d->alpha, d->beta, scores, prior, fused);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "fuse/pool launch");
@@ -360,7 +369,8 @@ int cc_fuse_prior_pool(cc_ctx* ctx, const cc_layer_desc* desc, const float* scor
   Plan p;
   int rc = build_plan(ctx, desc, &p);
   if (rc != CC_OK) return rc;
-  if (!scores || !prior || !fused) return fail(ctx, CC_ERR_INVALID_ARG, "NULL tensor pointer");
+  if ((!scores && desc->fill_mode != CC_FILL_NEAREST) || !prior || !fused)
+    return fail(ctx, CC_ERR_INVALID_ARG, "NULL tensor pointer");
   return run_fuse(ctx, desc, p, scores, prior, fused, stream);
 }
 
@@ -425,9 +435,10 @@ int cc_compress_layer(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win,
   char* w = (char*)ws;
   float* scores = (float*)(w + p.off_scores);
   float* fused = (float*)(w + p.off_fused);
-  if ((rc = run_score(ctx, desc, p, q_win, k, scores, nullptr, w, stream)) != CC_OK) return rc;
+  const bool nearest = desc->fill_mode == CC_FILL_NEAREST;   // the scores play no part then
+  if (!nearest && (rc = run_score(ctx, desc, p, q_win, k, scores, nullptr, w, stream)) != CC_OK) return rc;
   const int cluster = select_cluster_size(p.bt, p.g.hkv);
-  if (cluster > 0) {
+  if (cluster > 0 && !nearest) {
     rc = run_fuse_select(ctx, desc, p, cluster, scores, prior, fused, idx, count, stream);
     if (rc != CC_OK) return rc;
   } else {

@@ -121,6 +121,10 @@ cudaError_t launch_score_tc(const Launch& L, const BatchTable& bt, const Geometr
                             const void* q, const void* k, float* scores, float* lse, void* ws,
                             void* encode_fn, int64_t pool_rows, int* drv_err);
 
+// fused[h][j] = -(distance of token j to the closest token with prior >= threshold), every head
+cudaError_t launch_nearest_fill(const Launch& L, const BatchTable& bt, const Geometry& g,
+                                float force_threshold, const float* prior, float* fused);
+
 cudaError_t launch_fuse_pool(const Launch& L, const BatchTable& bt, const Geometry& g,
                              int pool_kind, int pool_size, float alpha, float beta,
                              const float* scores, const float* prior, float* fused);

@@ -60,7 +60,66 @@ fuse_pool_kernel(const __grid_constant__ BatchTable bt, int pool_kind, int pool_
   }
 }
 
+// Nearest-to-protected fill (Section 4.4, last sentence of "Token-level protection"): one CTA per
+// sequence.  Every thread owns a contiguous segment of the tokens; the position of the last
+// protected token before a segment and of the first one after it come from two block-wide scans,
+// then each thread sweeps its segment forwards and backwards.  The value, minus the distance to
+// the closest protected token (minus n when there is none), is the same for every head: it is
+// computed into head 0's row and copied to the others.
+constexpr int kNearThreads = 1024;
+
+__global__ void __launch_bounds__(kNearThreads)
+nearest_fill_kernel(const __grid_constant__ BatchTable bt, int hkv, float theta,
+                    const float* __restrict__ prior, float* __restrict__ fused) {
+  __shared__ int s_last[kNearThreads], s_first[kNearThreads];
+  const int s = blockIdx.x;
+  const SeqInfo& q = bt.seq[s];
+  const int n = q.n;
+  if (n == 0) return;
+  const float* p = prior + q.tok_off;
+  float* f0 = fused + q.item_off;
+  const int t = threadIdx.x;
+  const int seg = (n + kNearThreads - 1) / kNearThreads;
+  const int lo = min(n, t * seg), hi = min(n, lo + seg);
+  int last = -1, first = n + n;              // "none": far enough that the distance exceeds n
+  for (int j = lo; j < hi; ++j)
+    if (p[j] >= theta) { last = j; if (first > n) first = j; }
+  s_last[t] = last;
+  s_first[t] = first;
+  __syncthreads();
+  // inclusive scans: maximum of `last` over the threads up to t, minimum of `first` from t on
+  for (int d = 1; d < kNearThreads; d <<= 1) {
+    const int a = t >= d ? s_last[t - d] : -1;
+    const int b = t + d < kNearThreads ? s_first[t + d] : n + n;
+    __syncthreads();
+    s_last[t] = max(s_last[t], a);
+    s_first[t] = min(s_first[t], b);
+    __syncthreads();
+  }
+  int before = t > 0 ? s_last[t - 1] : -1;                       // last protected token before lo
+  const int after = t + 1 < kNearThreads ? s_first[t + 1] : n + n;   // first one at or after hi
+  for (int j = lo; j < hi; ++j) {
+    if (p[j] >= theta) before = j;
+    f0[j] = before >= 0 ? (float)(j - before) : (float)n;
+  }
+  int next = after;
+  for (int j = hi - 1; j >= lo; --j) {
+    if (p[j] >= theta) next = j;
+    const float d = next < n ? (float)(next - j) : (float)n;
+    f0[j] = -fminf(f0[j], d);
+  }
+  __syncthreads();
+  for (int h = 1; h < hkv; ++h)
+    for (int j = t; j < n; j += kNearThreads) fused[(int64_t)h * bt.m_tot + q.item_off + j] = f0[j];
+}
+
 }  // namespace
+
+cudaError_t launch_nearest_fill(const Launch& L, const BatchTable& bt, const Geometry& g,
+                                float force_threshold, const float* prior, float* fused) {
+  nearest_fill_kernel<<<bt.num_seqs, kNearThreads, 0, L.stream>>>(bt, g.hkv, force_threshold, prior, fused);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_fuse_pool(const Launch& L, const BatchTable& bt, const Geometry& g,
                              int pool_kind, int pool_size, float alpha, float beta,

@@ -53,6 +53,8 @@ class Workload:
     span_ratio: float = 0.0          # 0 = no cap on forced tokens
     span_min: int = 16
     causal: bool = False             # window = last w tokens of the sequence itself (masked)
+    fill_mode: int = 0               # 1 = the budget left by the protected tokens goes to their nearest neighbours
+    seq_budgets: Tuple[int, ...] = ()   # ragged batch: explicit per-sequence budgets (else budget_frac)
 
     @property
     def group(self) -> int:
@@ -64,6 +66,8 @@ class Workload:
 
     @property
     def budgets(self) -> Tuple[int, ...]:
+        if self.seq_budgets:
+            return self.seq_budgets
         if self.seq_lens:
             return tuple(int(np.floor(self.budget_frac * s)) for s in self.seq_lens)
         return (self.budget,)

@@ -39,7 +39,7 @@ def desc_for(wl: gen.Workload, mode: int, page_table=None, out_pt_stride: int = 
               force_threshold=wl.force_threshold if force else math.inf,
               span_ratio=wl.span_ratio, span_min=wl.span_min, page_size=wl.page_size,
               page_table=page_table, out_page_table_stride=out_pt_stride,
-              pool_pages=pool_pages, causal=wl.causal)
+              pool_pages=pool_pages, causal=wl.causal, fill_mode=wl.fill_mode)
     if wl.seq_lens:
         return cc.Desc(wl.n_heads_q, wl.n_heads_kv, wl.window, seq_lens=wl.lens,
                        budgets=wl.budgets, **kw)

@@ -63,8 +63,10 @@ def check_layer(wl, x, mode, tol):
         prior = x.prior[lo:lo + n]
         ref = orc.compress_sequence(x.q_win[s], k_s, v_s, prior, wl.n_heads_kv, wl.pool_kind,
                                     wl.pool_size, b, wl.alpha, wl.beta, wl.force_threshold,
-                                    wl.span_ratio, wl.span_min, chunk, causal=wl.causal)
-        assert_scores_close(got["scores"][:, lo:lo + n], ref["scores"], rows, n, tol)
+                                    wl.span_ratio, wl.span_min, chunk, causal=wl.causal,
+                                    nearest_fill=bool(wl.fill_mode))
+        if not wl.fill_mode:                  # (the nearest-token fill does not compute scores)
+            assert_scores_close(got["scores"][:, lo:lo + n], ref["scores"], rows, n, tol)
         m = len(ref["item_prior"])
         # the protected set (capped to the span budget when a span ratio is set) depends on the
         # prior alone, so it is taken from the oracle; what the scores decide is checked below
@@ -82,6 +84,9 @@ def check_layer(wl, x, mode, tol):
         # ... plus the rounding of the kernels' fp32 fusion (two products and a sum, half an ulp
         # each) against the fp64 reference: it decides the order when beta * p dominates
         band = abs(wl.alpha) * band_u * 2 + 1e-12 + 3 * 2.0 ** -24 * np.abs(ref["fused"])
+        if wl.fill_mode:
+            band = np.zeros_like(ref["fused"])          # distances are integers: nothing to forgive
+            np.testing.assert_array_equal(got["fused"][:, off_i:off_i + m], ref["fused"])
         for h in range(wl.n_heads_kv):
             assert got["count"][s, h] == keep
             idx = got["idx"][h, off_b:off_b + keep]
@@ -183,3 +188,16 @@ def test_more_items_than_a_cluster_holds():
     ref = orc.select_tokens(fused[0], x.prior, wl.n, wl.budget, wl.force_threshold, 0.5, 16)
     assert count[0] == len(ref) == wl.budget
     np.testing.assert_array_equal(idx[0, :len(ref)], ref)
+
+
+@pytest.mark.parametrize("mode,tol", MODES)
+def test_nearest_token_fill_through_the_fused_call(mode, tol):
+    """Section 4.4, last sentence of "Token-level protection": the budget left by the protected
+    tokens goes to the tokens nearest to them; bit for bit (the ranking values are integers)."""
+    from dataclasses import replace
+    wl = replace(gen.workloads()["tiny"], fill_mode=cc.CC_FILL_NEAREST)
+    check_layer(wl, gen.make_layer(wl, layer=11), mode, tol)
+    wl = gen.Workload("rpnear", 37, 1, 8, 2, 128, 16, gen.POOL_AVG, 5, 0,
+                      seq_lens=(700, 40, 2050, 129, 5000), budget_frac=0.3, page_size=16,
+                      span_ratio=0.5, span_min=16, fill_mode=cc.CC_FILL_NEAREST)
+    check_layer(wl, gen.make_layer(wl), mode, tol)

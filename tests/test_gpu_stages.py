@@ -395,3 +395,21 @@ def test_exp_rate_probe_reports_a_plausible_rate():
     assert 12.0 < reg < 40.0, reg
     assert 8.0 < tm < 40.0, tm
     assert ctx().poll() == 0
+
+
+@pytest.mark.parametrize("n", [1, 31, 1024, 1025, 5000, 70001])
+@pytest.mark.parametrize("density", [0.0, 0.002, 0.07, 1.0])
+def test_nearest_fill_values_bit_exact(n, density):
+    """cc_fuse_prior_pool with CC_FILL_NEAREST against the oracle's two-sweep distances."""
+    rng = np.random.Generator(np.random.PCG64(n + int(1000 * density)))
+    prior = (rng.random(n) < density).astype(np.float32)
+    hkv = 3
+    d = cc.Desc(hkv, hkv, 4, n=n, budget=max(1, n // 10), pool_kind=cc.CC_POOL_NONE, pool_size=1,
+                force_threshold=0.5, fill_mode=cc.CC_FILL_NEAREST)
+    fused_c, full = guarded((hkv, n), torch.float32, -77.0)
+    cc.cc_fuse_prior_pool(ctx(), d, None, f32_dev(prior), fused_c)
+    assert ctx().poll() == 0
+    assert guards_intact(full, -77.0)
+    ref = orc.nearest_fill_values(prior, 0.5).astype(np.float32)
+    for h in range(hkv):
+        np.testing.assert_array_equal(fused_c[h].cpu().numpy(), ref)
