@@ -243,6 +243,9 @@ def bench_config(wl, n_sets, set_bytes):
 
 
 # ----------------------------------------------------------------------------- CUDA arm
+PRIOR_OVERRIDE = {}       # workloads whose prior comes from the planner instead of the generator
+
+
 def bench_workloads():
     """Every configuration of the benchmark table, in the order reported."""
     from paper_2604_10235_b200 import inputs as gen
@@ -251,6 +254,12 @@ def bench_workloads():
     table = [w["tiny"], w["llama3_8b"]]
     table += [gen.qwen_variant(q, b, "15") for b in (1024, 4096, 8192)]
     table += [w["chunk10"], w["ragged_paged"], w["paper_avg5_w128"]]
+    # the paper's own configuration as a planned ragged batch, at both capacities of the paper
+    from paper_2604_10235_b200 import planning
+    for capacity in (0.4, 0.6):
+        wl, prior = planning.paper_chunks(capacity)
+        PRIOR_OVERRIDE[wl.name] = prior
+        table.append(wl)
     return {x.name: x for x in table}
 
 
@@ -277,6 +286,8 @@ class WorkloadRun:
         self.dev_sets, self.host_sets = [], []
         for i, layer in enumerate(layers):
             x = layout0 if (i == 0 and layout0 is not None) else gen.make_layer(wl, layer=layer)
+            if wl.name in PRIOR_OVERRIDE:
+                x.prior = PRIOR_OVERRIDE[wl.name]
             if rank == 0 and i == 0:
                 _ORACLE_INPUTS.setdefault(wl.name, x)     # layer 0: what the CPU baseline runs on
             if wl.page_size and i > 0:

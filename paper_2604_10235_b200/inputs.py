@@ -250,3 +250,44 @@ def small_case(seed: int, n: int, window: int, n_heads_q: int, n_heads_kv: int,
     k = rng.standard_normal((n, n_heads_kv, head_dim), dtype=np.float32)
     v = rng.standard_normal((n, n_heads_kv, head_dim), dtype=np.float32)
     return f32_to_bf16_bits(q), f32_to_bf16_bits(k), f32_to_bf16_bits(v)
+
+
+@dataclass
+class ChunkBatch:
+    """Synthetic retrieved chunks of one request, as the planner sees them (Sections 4.3, 4.4):
+    lengths, chunk-level structural scores, and per chunk the structural spans (half-open token
+    ranges with an importance score and a protected flag for signatures / query matches)."""
+
+    lens: Tuple[int, ...]
+    sigma: np.ndarray                      # [chunks] float64 in [0, 1]
+    spans: List[Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]]   # starts, ends, scores, protected
+
+
+def chunk_batch(seed: int, count: int = 32, lo: int = 128, hi: int = 4096) -> ChunkBatch:
+    """``count`` chunks of ``lo``..``hi`` tokens (Appendix "Compression settings": method-level
+    chunks of at most 4096 tokens).  Spans: one per structural line of the chunk's seeded
+    line-label layout, from the line's first token over a local context of 6 to 40 tokens (spans
+    overlap, and together cover more tokens than a span budget admits); the score is the
+    label's weight of the appendix (call .20, branch .18, return .14, assignment .14) plus a
+    seeded term below .24 standing for the query-alignment and def-use terms; the first line of
+    a chunk (the signature) and about 3 % of the others are protected."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    lens = tuple(int(x) for x in rng.integers(lo, hi + 1, size=count))
+    sigma = rng.random(count)
+    weight = {0: 0.20, 1: 0.18, 2: 0.14, 3: 0.14}
+    spans = []
+    for c, n in enumerate(lens):
+        _, label = structural_prior(seed * 1000 + c, n)
+        starts, ends, scores, prot = [0], [min(n, 8)], [0.5], [True]       # the signature line
+        line_start = np.flatnonzero(np.diff(np.concatenate([[-1], label.astype(np.int64)])) != 0)
+        for j in line_start:
+            lab = int(label[j])
+            if lab == len(LABELS) - 1 or j == 0:
+                continue
+            starts.append(int(j))
+            ends.append(int(min(n, j + rng.integers(6, 41))))
+            scores.append(weight[lab] + float(rng.random()) * 0.24)
+            prot.append(bool(rng.random() < 0.03))
+        spans.append((np.asarray(starts, np.int32), np.asarray(ends, np.int32),
+                      np.asarray(scores, np.float32), np.asarray(prot, bool)))
+    return ChunkBatch(lens, sigma, spans)

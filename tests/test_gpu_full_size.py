@@ -63,3 +63,15 @@ def test_llama_shape_selection_with_span_cap_full_size(ratio, smin):
         ref = orc.select_tokens(fused[h], x.prior, wl.n, wl.budget, wl.force_threshold, ratio, smin)
         assert count[h] == len(ref) == wl.budget
         np.testing.assert_array_equal(idx[h, :len(ref)], ref)
+
+
+@pytest.mark.parametrize("capacity", [0.4, 0.6])
+def test_paper_configuration_as_a_planned_ragged_batch(capacity):
+    """The paper's own setting end to end: 32 chunks of up to 4096 tokens, budgets from
+    cc_plan_budgets, protected tokens from cc_select_spans, average pooling 5, window 128, span
+    ratio 0.5 / minimum 16 active, one ragged cc_compress_layer call against the oracle."""
+    from paper_2604_10235_b200 import planning
+    wl, prior = planning.paper_chunks(capacity)
+    x = gen.make_layer(wl, layer=1)
+    x.prior = prior
+    check_layer(wl, x, cc.CC_MODE_BF16, 2e-3)

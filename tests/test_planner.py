@@ -83,3 +83,25 @@ def test_planned_protection_feeds_the_selection():
     fused = rng.random(n).astype(np.float32)
     kept = orc.select_tokens(fused, mask.astype(np.float32), n, budget, 0.5, 0.0, 0, 1)
     assert set(np.flatnonzero(mask)) <= set(kept.tolist())
+
+
+@pytest.mark.parametrize("capacity", [0.4, 0.6])
+def test_planned_chunk_batch_matches_the_oracle(capacity):
+    """Budgets and protected-token masks of a 32-chunk batch, as `planning.plan_chunk_batch` hands
+    them to the compression call, against the oracle's planner (Sections 4.3 and 4.4)."""
+    from paper_2604_10235_b200 import inputs as gen
+    from paper_2604_10235_b200 import planning
+    cb = gen.chunk_batch(5005)
+    budgets, prior = planning.plan_chunk_batch(cb.lens, cb.sigma, cb.spans, capacity)
+    ref_b, _ = orc.plan_budgets(cb.sigma, cb.lens, capacity, 1.0, 0.5, 1.5, 1e-6)
+    assert list(budgets) == ref_b.tolist()
+    off, binding_caps = 0, 0
+    for n, b, (st, en, sc, pr) in zip(cb.lens, budgets, cb.spans):
+        ref_mask, _ = orc.select_spans(st, en, sc, pr, n, b, 0.5, 16)
+        assert np.array_equal(prior[off:off + n] > 0, ref_mask)
+        binding_caps += int(ref_mask.sum() >= orc.span_budget(b, 0.5, 16))
+        off += n
+    assert off == len(prior)
+    assert binding_caps >= len(cb.lens) // 2          # the span budget is what limits most chunks
+    wl, p2 = planning.paper_chunks(capacity)
+    assert wl.lens == cb.lens and wl.budgets == budgets and np.array_equal(p2, prior)
