@@ -687,7 +687,9 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
           const bool masked_tile = CAUSAL && key0 + kTileKeys > n_cur - g.window + 1;
           auto drain = [&](auto masked) {
           constexpr bool kMasked = decltype(masked)::value;
-          int valid_r = valid;
+          // a warp whose 32 rows all lie past the padded window (last row block of a row count
+          // that is not a multiple of 128) has nothing to sum: it only hands the buffer back
+          int valid_r = sub * 128 + quad * 32 >= P.rows_pad ? 0 : valid;
           if (kMasked) {
             const int t_row = (sub * 128 + row_in_tile) / g.group;
             if (t_row < g.window) valid_r = min(valid, n_cur - g.window + t_row + 1 - key0);
