@@ -485,7 +485,7 @@ def run_ours(args, wl):
     h2d, d2h = comp.h2d_bytes, comp.d2h_bytes
     n_sets_head, set_bytes_head = run.n_sets, run.set_bytes
 
-    table, aux, cpu = None, None, None
+    table, aux, cpu, host = None, None, None, None
     if rank == 0 and world == 1 and not args.no_table:
         table = {wl.name: head}
         del run, comp, graph
@@ -498,6 +498,7 @@ def run_ours(args, wl):
             del r
             torch.cuda.empty_cache()
         aux = chunk_scoring_bandwidth(ctx, peaks)
+        host = host_time_per_layer(ctx, rank)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = oracle_throughput(wl, 12.0)
         cpu.pop("seconds", None)
@@ -522,6 +523,7 @@ def run_ours(args, wl):
             "ms_per_step_warm_l2": head["ms_per_step_warm_l2"],
             "workloads": table,
             "chunk_scoring": aux,
+            "host_time_tiny_no_graph": host,
             "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": n_e2e},
@@ -533,6 +535,45 @@ def run_ours(args, wl):
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def host_time_per_layer(ctx, rank):
+    """Host time of enqueueing one layer of the tiny workload (whose GPU time is below it) without
+    a CUDA graph: one cc_compress_layer call per layer against one cc_compress_layers call for 32
+    layers.  Wall clock around the enqueue loop, stream synchronised before and after."""
+    import torch
+    from paper_2604_10235_b200 import binding as cc
+    from paper_2604_10235_b200 import inputs as gen
+    r = WorkloadRun(ctx, gen.workloads()["tiny"], rank, pinned=False)
+    comp, sets, n = r.comp, r.dev_sets, 32
+    layers = [sets[i % len(sets)] for i in range(n)]
+    outs_k = [torch.empty_like(comp.k_out) for _ in range(n)]
+    outs_v = [torch.empty_like(comp.v_out) for _ in range(n)]
+    idxs = [torch.empty_like(comp.idx) for _ in range(n)]
+    cnts = [torch.empty_like(comp.count) for _ in range(n)]
+    out = {}
+    for name in ("per_call", "all_layers"):
+        best = None
+        for _ in range(5):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            if name == "per_call":
+                for l, (q, k, v, p) in enumerate(layers):
+                    cc.cc_compress_layer(ctx, comp.desc, q, k, v, p, outs_k[l], outs_v[l], idxs[l], cnts[l],
+                                         ws=comp.ws)
+            else:
+                cc.cc_compress_layers(ctx, comp.desc, [x[0] for x in layers], [x[1] for x in layers],
+                                      [x[2] for x in layers], layers[0][3], outs_k, outs_v, idxs, cnts,
+                                      ws=comp.ws)
+            t1 = time.perf_counter()
+            torch.cuda.synchronize()
+            t2 = time.perf_counter()
+            cur = ((t1 - t0) / n * 1e6, (t2 - t0) / n * 1e6)
+            best = cur if best is None or cur[1] < best[1] else best
+        out[name] = {"enqueue_us_per_layer": best[0], "wall_us_per_layer": best[1]}
+    if ctx.poll() != 0:
+        raise RuntimeError("device status after the host-time measurement")
+    return out
 
 
 def chunk_scoring_bandwidth(ctx, peaks):

@@ -202,6 +202,20 @@ int cc_compress_layer(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win,
                       int32_t* idx, int32_t* count, const int32_t* free_pages,
                       int32_t* out_page_table, void* ws, size_t ws_bytes, void* stream);
 
+/* The same step for n_layers layers of one batch, enqueued back to back (Section 4.5: every layer
+ * is compressed on its own, with the same geometry and the same prior).  q_win, k, v, k_out,
+ * v_out, idx, count (and, for the paged layout, free_pages and out_page_table; NULL otherwise)
+ * are HOST arrays of n_layers device pointers, entry l being what cc_compress_layer takes for
+ * layer l.  The descriptor is checked and the workspace carved once; the layers share the
+ * workspace (they run one after the other on the stream), so the intermediates left in it are
+ * those of the last layer.  Results are those of n_layers separate calls, bit for bit. */
+int cc_compress_layers(cc_ctx* ctx, const cc_layer_desc* desc, int32_t n_layers,
+                       const void* const* q_win, const void* const* k, const void* const* v,
+                       const float* prior, void* const* k_out, void* const* v_out,
+                       int32_t* const* idx, int32_t* const* count,
+                       const int32_t* const* free_pages, int32_t* const* out_page_table,
+                       void* ws, size_t ws_bytes, void* stream);
+
 /* Str. Score (Section 5.3, caption of the bug-localization table): the share of the structurally
  * critical tokens that survives compression, which the paper averages over layers and chunks.
  * For every sequence s and

@@ -32,7 +32,7 @@ EXPORTS = ("cc_create", "cc_destroy", "cc_status_string", "cc_last_error", "cc_p
            "cc_workspace_bytes", "cc_score_window", "cc_fuse_prior_pool", "cc_topk_select",
            "cc_compact_kv", "cc_compress_layer", "cc_workspace_views", "cc_topk_select_static",
            "cc_structural_score", "cc_plan_budgets", "cc_select_spans", "cc_ppl_chunk_scores",
-           "cc_select_chunks", "cc_exp_rate_probe")
+           "cc_select_chunks", "cc_exp_rate_probe", "cc_compress_layers")
 CC_STATIC_SELECT_MAX_ITEMS = 1 << 20
 
 
@@ -104,6 +104,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
                                     C.c_int32, vp, vp, vp]
     lib.cc_compress_layer.argtypes = [vp, dp] + [vp] * 10 + [vp, sz, vp]
     lib.cc_exp_rate_probe.argtypes = [vp, C.c_int32, C.c_int32, C.POINTER(C.c_double), vp]
+    lib.cc_compress_layers.argtypes = [vp, dp, C.c_int32] + [vp] * 3 + [vp] + [vp] * 6 + [vp, sz, vp]
     lib.cc_workspace_views.argtypes = [vp, dp, vp, C.POINTER(vp), C.POINTER(vp)]
     for name in EXPORTS:
         if name not in ("cc_status_string", "cc_last_error", "cc_workspace_bytes"):
@@ -366,6 +367,26 @@ def cc_exp_rate_probe(ctx: Context, from_tmem: bool, iters: int = 4000, stream=N
     ctx.check(ctx.lib.cc_exp_rate_probe(ctx.handle, 1 if from_tmem else 0, iters, C.byref(rate),
                                         _stream(stream)))
     return float(rate.value)
+
+
+def _ptr_array(tensors):
+    """Host array of the device pointers of a list of tensors (None -> NULL array)."""
+    if tensors is None:
+        return None
+    arr = (C.c_void_p * len(tensors))(*[t.data_ptr() for t in tensors])
+    return arr
+
+
+def cc_compress_layers(ctx: Context, desc: Desc, q_win, k, v, prior, k_out, v_out, idx, count,
+                       free_pages=None, out_page_table=None, ws=None, stream=None):
+    """cc_compress_layer for a list of layers in one call: every tensor argument except ``prior``
+    and ``ws`` is a list with one tensor per layer."""
+    ws = ctx.workspace(desc) if ws is None else ws
+    n = len(k)
+    arrays = [_ptr_array(x) for x in (q_win, k, v)]
+    outs = [_ptr_array(x) for x in (k_out, v_out, idx, count, free_pages, out_page_table)]
+    ctx.check(ctx.lib.cc_compress_layers(ctx.handle, C.byref(desc.c), n, *arrays, _ptr(prior), *outs,
+                                         _ptr(ws), ws.numel(), _stream(stream)))
 
 
 def cc_workspace_views(ctx: Context, desc: Desc, ws: torch.Tensor):

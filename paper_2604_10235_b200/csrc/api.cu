@@ -419,20 +419,19 @@ int cc_compact_kv(cc_ctx* ctx, const cc_layer_desc* desc, const void* k, const v
   return run_compact(ctx, desc, p, k, v, idx, k_out, v_out, free_pages, out_page_table, stream);
 }
 
-int cc_compress_layer(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win, const void* k,
-                      const void* v, const float* prior, void* k_out, void* v_out, int32_t* idx,
-                      int32_t* count, const int32_t* free_pages, int32_t* out_page_table,
-                      void* ws, size_t ws_bytes, void* stream) {
-  Plan p;
-  int rc = build_plan(ctx, desc, &p);
-  if (rc != CC_OK) return rc;
+namespace {
+
+// One layer of the fused step with a plan that is already built and checked.
+int compress_one(cc_ctx* ctx, const cc_layer_desc* desc, const Plan& p, const void* q_win,
+                 const void* k, const void* v, const float* prior, void* k_out, void* v_out,
+                 int32_t* idx, int32_t* count, const int32_t* free_pages, int32_t* out_page_table,
+                 char* w, void* stream) {
   if (!q_win || !k || !v || !prior || !count || (p.bt.b_tot > 0 && (!k_out || !v_out || !idx)))
     return fail(ctx, CC_ERR_INVALID_ARG, "NULL tensor pointer");
   if ((uintptr_t)q_win % 16 || (uintptr_t)k % 16 || (uintptr_t)v % 16 || (uintptr_t)k_out % 16 ||
       (uintptr_t)v_out % 16)
     return fail(ctx, CC_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned");
-  if ((rc = check_ws(ctx, p, ws, ws_bytes)) != CC_OK) return rc;
-  char* w = (char*)ws;
+  int rc;
   float* scores = (float*)(w + p.off_scores);
   float* fused = (float*)(w + p.off_fused);
   const bool nearest = desc->fill_mode == CC_FILL_NEAREST;   // the scores play no part then
@@ -447,6 +446,45 @@ int cc_compress_layer(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win,
   }
   if (p.bt.b_tot == 0) return CC_OK;
   return run_compact(ctx, desc, p, k, v, idx, k_out, v_out, free_pages, out_page_table, stream);
+}
+
+}  // namespace
+
+int cc_compress_layer(cc_ctx* ctx, const cc_layer_desc* desc, const void* q_win, const void* k,
+                      const void* v, const float* prior, void* k_out, void* v_out, int32_t* idx,
+                      int32_t* count, const int32_t* free_pages, int32_t* out_page_table,
+                      void* ws, size_t ws_bytes, void* stream) {
+  Plan p;
+  int rc = build_plan(ctx, desc, &p);
+  if (rc != CC_OK) return rc;
+  if ((rc = check_ws(ctx, p, ws, ws_bytes)) != CC_OK) return rc;
+  return compress_one(ctx, desc, p, q_win, k, v, prior, k_out, v_out, idx, count, free_pages,
+                      out_page_table, (char*)ws, stream);
+}
+
+int cc_compress_layers(cc_ctx* ctx, const cc_layer_desc* desc, int32_t n_layers,
+                       const void* const* q_win, const void* const* k, const void* const* v,
+                       const float* prior, void* const* k_out, void* const* v_out,
+                       int32_t* const* idx, int32_t* const* count,
+                       const int32_t* const* free_pages, int32_t* const* out_page_table,
+                       void* ws, size_t ws_bytes, void* stream) {
+  Plan p;
+  int rc = build_plan(ctx, desc, &p);
+  if (rc != CC_OK) return rc;
+  if (n_layers < 0) return fail(ctx, CC_ERR_INVALID_ARG, "negative layer count");
+  if (n_layers == 0) return CC_OK;
+  if (!q_win || !k || !v || !k_out || !v_out || !idx || !count)
+    return fail(ctx, CC_ERR_INVALID_ARG, "NULL pointer array");
+  if (p.bt.page_size > 0 && (!free_pages || !out_page_table))
+    return fail(ctx, CC_ERR_INVALID_ARG, "paged compaction needs free_pages and out_page_table");
+  if ((rc = check_ws(ctx, p, ws, ws_bytes)) != CC_OK) return rc;
+  for (int l = 0; l < n_layers; ++l) {
+    rc = compress_one(ctx, desc, p, q_win[l], k[l], v[l], prior, k_out[l], v_out[l], idx[l], count[l],
+                      free_pages ? free_pages[l] : nullptr, out_page_table ? out_page_table[l] : nullptr,
+                      (char*)ws, stream);
+    if (rc != CC_OK) return rc;
+  }
+  return CC_OK;
 }
 
 int cc_structural_score(cc_ctx* ctx, const cc_layer_desc* desc, const int32_t* idx,

@@ -66,3 +66,53 @@ def test_back_to_back_calls_match_single_calls(wl):
             assert torch.equal(got, exp)
     for got, exp in zip(_snapshot(shared), want[-1]):          # the last call through the shared one
         assert torch.equal(got, exp)
+
+
+def test_all_layers_call_equals_separate_calls():
+    """cc_compress_layers on three layers: indices, counts and gathered K/V of every layer equal
+    those of three cc_compress_layer calls, bit for bit; contiguous and paged."""
+    from gpu_util import bf16_dev, ctx, desc_for
+    for wl in (gen.workloads()["tiny"],
+               gen.Workload("rp", 32, 1, 8, 2, 128, 16, gen.POOL_MAX, 7, 0,
+                            seq_lens=(300, 40, 2050, 129), budget_frac=0.1, page_size=16)):
+        paged = wl.page_size > 0
+        xs = [gen.make_layer(wl, layer=l) for l in range(3)]
+        if paged:
+            for x in xs[1:]:
+                gen.repage(x, xs[0])
+        pt = torch.from_numpy(xs[0].page_table).cuda() if paged else None
+        b_tot = sum(wl.budgets)
+        stride = max((b + 15) // 16 for b in wl.budgets) + 1 if paged else 0
+        d = desc_for(wl, cc.CC_MODE_BF16, page_table=pt, out_pt_stride=stride, pool_pages=xs[0].pool_pages)
+        ws = ctx().workspace(d)
+        prior = torch.from_numpy(xs[0].prior).cuda()
+
+        def fresh():
+            q = [bf16_dev(x.q_win) for x in xs]
+            k = [bf16_dev(x.k) for x in xs]
+            v = [bf16_dev(x.v) for x in xs]
+            idx = [torch.full((wl.n_heads_kv, b_tot), -9, dtype=torch.int32, device="cuda") for _ in xs]
+            cnt = [torch.full((len(wl.lens), wl.n_heads_kv), -9, dtype=torch.int32, device="cuda") for _ in xs]
+            if paged:
+                ko, vo = k, v
+                free = [torch.from_numpy(x.free_pages).cuda() for x in xs]
+                opt = [torch.full((len(wl.lens), stride), -9, dtype=torch.int32, device="cuda") for _ in xs]
+            else:
+                ko = [torch.zeros((b_tot, wl.n_heads_kv, 128), dtype=torch.bfloat16, device="cuda") for _ in xs]
+                vo = [torch.zeros_like(t) for t in ko]
+                free = opt = None
+            return q, k, v, ko, vo, idx, cnt, free, opt
+
+        a = fresh()
+        for l in range(3):
+            cc.cc_compress_layer(ctx(), d, a[0][l], a[1][l], a[2][l], prior, a[3][l], a[4][l], a[5][l],
+                                 a[6][l], a[7][l] if paged else None, a[8][l] if paged else None, ws)
+        b = fresh()
+        cc.cc_compress_layers(ctx(), d, b[0], b[1], b[2], prior, b[3], b[4], b[5], b[6], b[7], b[8], ws)
+        assert ctx().poll() == 0
+        for l in range(3):
+            for j in (3, 4, 5, 6):
+                assert torch.equal(a[j][l].view(torch.int16) if a[j][l].dtype == torch.bfloat16 else a[j][l],
+                                   b[j][l].view(torch.int16) if b[j][l].dtype == torch.bfloat16 else b[j][l])
+            if paged:
+                assert torch.equal(a[8][l], b[8][l])
