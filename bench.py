@@ -229,17 +229,25 @@ def run_reference(args, wl):
     print(json.dumps(line), flush=True)
 
 
-def bench_config(wl, n_sets, set_bytes):
-    """The ``config`` object of the JSON line: the same keys for both arms."""
-    cfg = {"workload": wl.name, "n": list(wl.lens), "heads_q": wl.n_heads_q,
-           "heads_kv": wl.n_heads_kv, "window": wl.window, "pool": [wl.pool_kind, wl.pool_size],
-           "budget": list(wl.budgets), "chunk": wl.chunk_size, "page_size": wl.page_size}
-    if n_sets is not None:
-        cfg["layers_cycled"] = n_sets
-        cfg["launch"] = f"CUDA graph of {n_sets} fused steps, replayed"
-        cfg["l2"] = (f"inputs larger than L2: {n_sets} layer sets of {set_bytes / 1e6:.0f} MB cycled, "
-                     f"no set reused within {(n_sets - 1) * set_bytes / 1e6:.0f} MB of traffic")
-    return cfg
+def bench_config(wl, n_sets=None, set_bytes=None):
+    """The ``config`` object of the JSON line: the same for both arms (the layer-set figures follow
+    from the workload alone)."""
+    n_sets = sets_for(wl)
+    ps = wl.page_size
+    if ps:
+        rows = (sum((n + ps - 1) // ps for n in wl.lens) + sum((b + ps - 1) // ps for b in wl.budgets) + 8) * ps
+    else:
+        rows = sum(wl.lens)
+    row = wl.head_dim * 2
+    set_bytes = (2 * rows * wl.n_heads_kv * row + len(wl.lens) * wl.window * wl.n_heads_q * row
+                 + 4 * sum(wl.lens))
+    return {"workload": wl.name, "n": list(wl.lens), "heads_q": wl.n_heads_q,
+            "heads_kv": wl.n_heads_kv, "window": wl.window, "pool": [wl.pool_kind, wl.pool_size],
+            "budget": list(wl.budgets), "chunk": wl.chunk_size, "page_size": wl.page_size,
+            "layers_cycled": n_sets,
+            "launch": f"CUDA graph of {n_sets} fused steps, replayed (the CPU oracle arm: plain calls)",
+            "l2": (f"inputs larger than L2: {n_sets} layer sets of {set_bytes / 1e6:.0f} MB cycled, "
+                   f"no set reused within {(n_sets - 1) * set_bytes / 1e6:.0f} MB of traffic")}
 
 
 # ----------------------------------------------------------------------------- CUDA arm
