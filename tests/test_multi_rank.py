@@ -75,3 +75,28 @@ def test_bench_launcher_starts_the_ranks_itself():
     assert len(lines) == 1                      # rank 0 alone prints
     assert lines[0]["n_gpus"] == 2 and lines[0]["steps"] == 3
     assert lines[0]["ms_per_step"] >= 2.0 / 3   # the slower rank's time (rank 1 adds 2 ms)
+
+
+def test_bench_roofline_arithmetic():
+    """The host arithmetic behind the benchmark's roofline figures, against hand values for the
+    Llama-shaped workload: K once + Q + prior + gathered rows; 2 w G d flops and w G exponentials
+    per (key, KV head)."""
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    sys.path.insert(0, root)
+    import bench
+    wl = gen.workloads()["llama3_8b"]
+    work = bench.algorithmic_work(wl)
+    assert work["tokens"] == 32768
+    assert work["flops"] == 2.0 * 64 * 4 * 128 * 32768 * 8                    # 17.18 GFLOP
+    assert work["exps"] == 64 * 4 * 32768 * 8                                 # 67.1 M per pass
+    k_bytes = 32768 * 8 * 256
+    assert work["bytes"] == k_bytes + 64 * 32 * 256 + 4 * 32768 + 4 * 2048 * 8 * 256 + 4 * 2048 * 8
+    peaks = {"hbm_gbs": 6532.9, "bf16_tflops": 1628.0}
+    r = bench.roofline_of(work, peaks, 62.0e-6, clock_mhz=1965.0)
+    assert r["bound"] == "hbm" and abs(r["t_roof_us"] - 12.95) < 0.01 and abs(r["t_flops_us"] - 10.55) < 0.01
+    assert abs(r["frac"] - 12.95 / 62.0) < 1e-3
+    rate = bench.EXP_RATE["registers"]
+    assert abs(r["exp_bound_us"] - 2 * 67108864 / (rate * 148 * 1965e6) * 1e6) < 1e-6
+    cfg = bench.bench_config(gen.workloads()["ragged_paged"])
+    assert cfg["workload"] == "ragged_paged" and cfg["layers_cycled"] == 2 and "larger than L2" in cfg["l2"]
