@@ -58,6 +58,10 @@ def check_layer(wl, x, mode, tol):
     off_b = off_i = 0
     for s, (n, b) in enumerate(zip(wl.lens, wl.budgets)):
         keep = min(n, b)
+        if n == 0:                               # an empty sequence keeps nothing
+            assert (got["count"][s] == 0).all() and (got["idx"][:, off_b:off_b + b] == -1).all()
+            off_b += b
+            continue
         k_s, v_s = seq_kv(x, s)
         lo = int(x.tok_offsets[s])
         prior = x.prior[lo:lo + n]
@@ -201,3 +205,23 @@ def test_nearest_token_fill_through_the_fused_call(mode, tol):
                       seq_lens=(700, 40, 2050, 129, 5000), budget_frac=0.3, page_size=16,
                       span_ratio=0.5, span_min=16, fill_mode=cc.CC_FILL_NEAREST)
     check_layer(wl, gen.make_layer(wl), mode, tol)
+
+
+@pytest.mark.parametrize("mode,tol", MODES)
+def test_nearest_fill_edge_batches(mode, tol):
+    """Empty and one-token sequences, a budget above the length, and a sequence without any
+    protected token, in one ragged batch with the nearest-token fill."""
+    wl = gen.Workload("nearedge", 38, 1, 8, 2, 128, 8, gen.POOL_MAX, 3, 0,
+                      seq_lens=(0, 1, 33, 500), seq_budgets=(4, 1, 40, 77),
+                      fill_mode=cc.CC_FILL_NEAREST)
+    x = gen.make_layer(wl)
+    x.prior[1:34] = 0.0                       # sequences 1 and 2 have no protected token
+    check_layer(wl, x, mode, tol)
+
+
+def test_all_layers_call_with_no_layers_is_a_no_op():
+    wl = gen.workloads()["tiny"]
+    d = desc_for(wl, cc.CC_MODE_BF16)
+    cc.cc_compress_layers(ctx(), d, [], [], [], torch.zeros(wl.n, device="cuda"), [], [], [], [],
+                          ws=ctx().workspace(d))
+    assert ctx().poll() == 0
