@@ -42,6 +42,39 @@ TIMED_BLOCKS = 50         # the block of --steps steps is timed this many times;
 # are the figures of an earlier run, used only if the probe is not run.
 EXP_RATE = {"registers": 22.0, "tmem": 17.5, "source": "earlier run"}
 SM_COUNT = 148
+SM_MAX_MHZ = 1965.0
+# Exponentials per clock per SM that the arithmetic units allow, from unit counts: 16 special-
+# function results and 128 fp32 FMA lanes per clock.  An exponential on the special-function
+# path also takes 2 FMA-lane operations (scale-and-shift of the logit, accumulation), one on the
+# polynomial path 10 (scale, clamp, three for the range reduction, three for the cubic, exponent
+# insertion, accumulation).  With a fraction p on the polynomial path both pipes are full when
+# (1 - p) / 16 = (2 (1 - p) + 10 p) / 128, p = 3/8: 16 / (5/8) = 25.6 per clock per SM.
+ALU_EXP_PER_CLK_SM = 25.6
+
+
+def score_kernel_roofline(work, peaks, score_seconds):
+    """Roofline of the score stage (the dominant kernels): the binding one of HBM bytes, tensor
+    flops and exponential arithmetic, each as time at its peak; the other two fractions beside."""
+    t_b = work["score_bytes"] / (peaks["hbm_gbs"] * 1e9)
+    t_f = work["flops"] / (peaks["bf16_tflops"] * 1e12)
+    alu_peak = ALU_EXP_PER_CLK_SM * SM_COUNT * SM_MAX_MHZ * 1e6          # exponentials per second
+    t_a = 2.0 * work["exps"] / alu_peak                                  # both passes evaluate each once
+    if t_a >= t_f and t_a >= t_b:
+        roof = {"bound": "alu", "achieved": 2.0 * work["exps"] / score_seconds / 1e9,
+                "peak": alu_peak / 1e9, "unit": "Gexp/s",
+                "peak_source": "unit counts: 16 SFU results + 128 FMA lanes per clock per SM, "
+                               "148 SMs, 1965 MHz (25.6 exponentials per clock per SM)"}
+    elif t_f >= t_b:
+        roof = {"bound": "tensor", "achieved": work["flops"] / score_seconds / 1e12,
+                "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "peak_source": f"{peaks['source']} bf16 burst"}
+    else:
+        roof = {"bound": "hbm", "achieved": work["score_bytes"] / score_seconds / 1e9,
+                "peak": peaks["hbm_gbs"], "unit": "GB/s", "peak_source": f"{peaks['source']} copy"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["frac_of"] = {"alu": t_a / score_seconds, "tensor": t_f / score_seconds,
+                       "hbm": t_b / score_seconds}
+    return roof
 
 # DRAM bytes (read + write) of the two launches of the score stage, per workload, from the ncu
 # captures summarised under profiles/ (counters taken on the kernel as it stands in this tree):
@@ -458,16 +491,7 @@ def run_ours(args, wl):
     head = run.table_entry(peaks, clock_mhz)
     stage_us = head["stage_us"]
     score_s = stage_us["score"] * 1e-6
-    t_b = work["score_bytes"] / (peaks["hbm_gbs"] * 1e9)
-    t_f = work["flops"] / (peaks["bf16_tflops"] * 1e12)
-    if t_f >= t_b:
-        roof = {"bound": "tensor", "achieved": work["flops"] / score_s / 1e12,
-                "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "peak_source": f"{peaks['source']} bf16 burst"}
-    else:
-        roof = {"bound": "hbm", "achieved": work["score_bytes"] / score_s / 1e9,
-                "peak": peaks["hbm_gbs"], "unit": "GB/s", "peak_source": f"{peaks['source']} copy"}
-    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof = score_kernel_roofline(work, peaks, score_s)
     roof["kernel"] = "score_tc_kernel<1> + score_tc_kernel<2> (the two launches of the score stage)"
     traffic = SCORE_TRAFFIC_BYTES.get(wl.name, {})
     roof["traffic"] = traffic.get("live")

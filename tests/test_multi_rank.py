@@ -98,5 +98,13 @@ def test_bench_roofline_arithmetic():
     assert abs(r["frac"] - 12.95 / 62.0) < 1e-3
     rate = bench.EXP_RATE["registers"]
     assert abs(r["exp_bound_us"] - 2 * 67108864 / (rate * 148 * 1965e6) * 1e6) < 1e-6
+    # dominant kernels: the binding one of bytes, flops and exponentials, each at its own peak
+    k = bench.score_kernel_roofline(work, dict(peaks, source="measured"), 50.0e-6)
+    t_alu = 2 * 67108864 / (25.6 * 148 * 1965e6)
+    assert k["bound"] == "alu" and abs(k["frac"] - t_alu / 50.0e-6) < 1e-9
+    assert abs(k["achieved"] - 2 * 67108864 / 50.0e-6 / 1e9) < 1e-6 and k["unit"] == "Gexp/s"
+    assert abs(k["frac_of"]["tensor"] - 10.55 / 50.0) < 1e-3 and abs(k["frac_of"]["hbm"] - 10.513 / 50.0) < 1e-4
+    slow_alu = dict(work, exps=work["exps"] / 100)        # without the exponentials the flops bind
+    assert bench.score_kernel_roofline(slow_alu, dict(peaks, source="measured"), 50.0e-6)["bound"] == "tensor"
     cfg = bench.bench_config(gen.workloads()["ragged_paged"])
     assert cfg["workload"] == "ragged_paged" and cfg["layers_cycled"] == 2 and "larger than L2" in cfg["l2"]
