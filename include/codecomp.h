@@ -190,7 +190,10 @@ int cc_topk_select_static(cc_ctx* ctx, const cc_layer_desc* desc, const float* f
  * taken in order from free_pages (device i32, sequences served in order), written to
  * out_page_table[s][.] (device i32, -1 padded).  k_out/v_out must not alias k/v rows that
  * are still to be read; in-place compaction is rejected when the pointers are equal and
- * the layout is contiguous. */
+ * the layout is contiguous.  k and v are only read here, 256 bytes per retained row: either may
+ * be page-locked host memory that the device can address (cudaHostAlloc, cudaHostRegister) instead
+ * of device memory, in which case only the retained rows cross the bus.  The same holds for v of
+ * cc_compress_layer and cc_compress_layers (k is read by the scoring and belongs on the device). */
 int cc_compact_kv(cc_ctx* ctx, const cc_layer_desc* desc, const void* k, const void* v,
                   const int32_t* idx, void* k_out, void* v_out,
                   const int32_t* free_pages, int32_t* out_page_table, void* stream);

@@ -135,9 +135,18 @@ class LayerCompressor:
         self.h_idx = torch.empty(self.idx.shape, dtype=torch.int32).pin_memory()
         self.h_count = torch.empty(self.count.shape, dtype=torch.int32).pin_memory()
 
+    def h2d_bytes_of(self, v_in_place: bool) -> int:
+        """Bytes that cross to the device per run_host call: Q, K and the prior, plus all of V or,
+        when V is gathered in place from page-locked host memory, only its retained rows."""
+        n = sum(t.numel() * t.element_size() for t in (self.q, self.k, self.prior))
+        if not v_in_place:
+            return n + self.v.numel() * self.v.element_size()
+        kept = sum(min(b, m) for b, m in zip(self.wl.budgets, self.wl.lens))
+        return n + kept * self.wl.n_heads_kv * self.wl.head_dim * self.v.element_size()
+
     @property
     def h2d_bytes(self) -> int:
-        return sum(t.numel() * t.element_size() for t in (self.q, self.k, self.v, self.prior))
+        return self.h2d_bytes_of(False)
 
     @property
     def d2h_bytes(self) -> int:
@@ -146,24 +155,34 @@ class LayerCompressor:
             outs.append(self.out_page_table)
         return sum(t.numel() * t.element_size() for t in outs)
 
-    def run_device(self, q, k, v, prior) -> None:
+    def run_device(self, q, k, v, prior, v_src=None) -> None:
         """Inputs already on the device; outputs land in self.k_out / v_out (contiguous) or in
-        fresh pages of k / v (paged), plus idx / count / out_page_table."""
+        fresh pages of k / v (paged), plus idx / count / out_page_table.  ``v_src`` (page-locked
+        host memory laid out like v) makes the compaction read the retained V rows from there."""
         if self.paged:
-            cc.cc_compress_layer(self.ctx, self.desc, q, k, v, prior, k, v, self.idx, self.count,
+            cc.cc_compress_layer(self.ctx, self.desc, q, k, v if v_src is None else v_src, prior,
+                                 k, v, self.idx, self.count,
                                  self.free_pages, self.out_page_table, ws=self.ws)
         else:
-            cc.cc_compress_layer(self.ctx, self.desc, q, k, v, prior, self.k_out, self.v_out,
-                                 self.idx, self.count, ws=self.ws)
+            cc.cc_compress_layer(self.ctx, self.desc, q, k, v if v_src is None else v_src, prior,
+                                 self.k_out, self.v_out, self.idx, self.count, ws=self.ws)
 
-    def run_host(self, q_h, k_h, v_h, prior_h) -> Dict[str, torch.Tensor]:
+    def run_host(self, q_h, k_h, v_h, prior_h, v_in_place: bool = False) -> Dict[str, torch.Tensor]:
         """Inputs in (pinned) host memory: copy in, compress, copy the compacted cache back.
-        Everything is enqueued on the current stream; the caller synchronises."""
+        Everything is enqueued on the current stream; the caller synchronises.
+
+        V takes no part in the scoring: with ``v_in_place`` (v_h page-locked) it is not copied;
+        the compaction kernel reads the retained rows of v_h across the bus and writes them to
+        the device-side result, which cuts the bytes copied in by almost half."""
         self.q.copy_(q_h, non_blocking=True)
         self.k.copy_(k_h, non_blocking=True)
-        self.v.copy_(v_h, non_blocking=True)
+        if v_in_place:
+            if not v_h.is_pinned() or v_h.shape != self.v.shape or not v_h.is_contiguous():
+                raise ValueError("v_in_place needs a contiguous page-locked tensor shaped like the V pool")
+        else:
+            self.v.copy_(v_h, non_blocking=True)
         self.prior.copy_(prior_h, non_blocking=True)
-        self.run_device(self.q, self.k, self.v, self.prior)
+        self.run_device(self.q, self.k, self.v, self.prior, v_src=v_h if v_in_place else None)
         out = {"k_out": self.h_k_out, "v_out": self.h_v_out, "idx": self.h_idx,
                "count": self.h_count}
         if self.paged:

@@ -245,11 +245,14 @@ def _stream(stream: Optional[int]) -> C.c_void_p:
     return C.c_void_p(stream)
 
 
-def _ptr(t: Optional[torch.Tensor]) -> C.c_void_p:
+def _ptr(t: Optional[torch.Tensor], pinned_ok: bool = False) -> C.c_void_p:
+    """Address of a CUDA tensor; with ``pinned_ok`` also of a page-locked host tensor (its address
+    is valid on the device: the V rows of a compaction may be gathered straight from it)."""
     if t is None:
         return C.c_void_p(0)
-    if not t.is_cuda:
-        raise ValueError("libcodecomp takes CUDA tensors only")
+    if not t.is_cuda and not (pinned_ok and t.is_pinned()):
+        raise ValueError("libcodecomp takes CUDA tensors only" +
+                         (" (or page-locked host memory here)" if pinned_ok else ""))
     return C.c_void_p(t.data_ptr())
 
 
@@ -284,7 +287,7 @@ def cc_topk_select_static(ctx: Context, desc: Desc, fused, prior, idx, count, st
 
 def cc_compact_kv(ctx: Context, desc: Desc, k, v, idx, k_out, v_out, free_pages=None,
                   out_page_table=None, stream=None):
-    ctx.check(ctx.lib.cc_compact_kv(ctx.handle, C.byref(desc.c), _ptr(k), _ptr(v), _ptr(idx),
+    ctx.check(ctx.lib.cc_compact_kv(ctx.handle, C.byref(desc.c), _ptr(k, True), _ptr(v, True), _ptr(idx),
                                     _ptr(k_out), _ptr(v_out), _ptr(free_pages),
                                     _ptr(out_page_table), _stream(stream)))
 
@@ -355,7 +358,7 @@ def cc_select_spans(starts, ends, scores, protected, n: int, budget: int, span_r
 def cc_compress_layer(ctx: Context, desc: Desc, q_win, k, v, prior, k_out, v_out, idx, count,
                       free_pages=None, out_page_table=None, ws=None, stream=None):
     ws = ctx.workspace(desc) if ws is None else ws
-    ctx.check(ctx.lib.cc_compress_layer(ctx.handle, C.byref(desc.c), _ptr(q_win), _ptr(k), _ptr(v),
+    ctx.check(ctx.lib.cc_compress_layer(ctx.handle, C.byref(desc.c), _ptr(q_win), _ptr(k), _ptr(v, True),
                                         _ptr(prior), _ptr(k_out), _ptr(v_out), _ptr(idx),
                                         _ptr(count), _ptr(free_pages), _ptr(out_page_table),
                                         _ptr(ws), ws.numel(), _stream(stream)))
