@@ -129,11 +129,15 @@ class LayerCompressor:
                              + torch.arange(ps, device=dev)[None, :]).reshape(-1)
             self.h_k_out = torch.empty((n_out_rows, hkv, d), dtype=bf).pin_memory()
             self.h_v_out = torch.empty((n_out_rows, hkv, d), dtype=bf).pin_memory()
+            self.k_stage = torch.empty((n_out_rows, hkv, d), dtype=bf, device=dev)
+            self.v_stage = torch.empty((n_out_rows, hkv, d), dtype=bf, device=dev)
         else:
             self.h_k_out = torch.empty(self.k_out.shape, dtype=bf).pin_memory()
             self.h_v_out = torch.empty(self.v_out.shape, dtype=bf).pin_memory()
         self.h_idx = torch.empty(self.idx.shape, dtype=torch.int32).pin_memory()
         self.h_count = torch.empty(self.count.shape, dtype=torch.int32).pin_memory()
+        self._side = None               # stream of the overlapped copies back to the host
+        self._readback_done = None      # event recorded after the last of them
 
     def h2d_bytes_of(self, v_in_place: bool) -> int:
         """Bytes that cross to the device per run_host call: Q, K and the prior, plus all of V or,
@@ -167,13 +171,20 @@ class LayerCompressor:
             cc.cc_compress_layer(self.ctx, self.desc, q, k, v if v_src is None else v_src, prior,
                                  self.k_out, self.v_out, self.idx, self.count, ws=self.ws)
 
-    def run_host(self, q_h, k_h, v_h, prior_h, v_in_place: bool = False) -> Dict[str, torch.Tensor]:
+    def run_host(self, q_h, k_h, v_h, prior_h, v_in_place: bool = False,
+                 overlap_readback: bool = False) -> Dict[str, torch.Tensor]:
         """Inputs in (pinned) host memory: copy in, compress, copy the compacted cache back.
         Everything is enqueued on the current stream; the caller synchronises.
 
         V takes no part in the scoring: with ``v_in_place`` (v_h page-locked) it is not copied;
         the compaction kernel reads the retained rows of v_h across the bus and writes them to
-        the device-side result, which cuts the bytes copied in by almost half."""
+        the device-side result, which cuts the bytes copied in by almost half.
+
+        With ``overlap_readback`` the copies back to the host run on a stream of the compressor's
+        own, so that they share the bus (which carries both directions at once) with the next
+        call's copies in; the next call's kernels wait for them before they overwrite the device
+        results.  Call ``finish()`` (or synchronise the device) before reading the host tensors."""
+        main = torch.cuda.current_stream()
         self.q.copy_(q_h, non_blocking=True)
         self.k.copy_(k_h, non_blocking=True)
         if v_in_place:
@@ -182,18 +193,41 @@ class LayerCompressor:
         else:
             self.v.copy_(v_h, non_blocking=True)
         self.prior.copy_(prior_h, non_blocking=True)
+        if self._readback_done is not None:          # the previous call's results are still going out
+            main.wait_event(self._readback_done)
+            self._readback_done = None
         self.run_device(self.q, self.k, self.v, self.prior, v_src=v_h if v_in_place else None)
         out = {"k_out": self.h_k_out, "v_out": self.h_v_out, "idx": self.h_idx,
                "count": self.h_count}
         if self.paged:
-            # the retained rows sit in the fresh pages of the pool: bring just those back
-            self.h_k_out.copy_(self.k[self.out_rows], non_blocking=True)
-            self.h_v_out.copy_(self.v[self.out_rows], non_blocking=True)
-            self.h_out_page_table.copy_(self.out_page_table, non_blocking=True)
+            # the retained rows sit in the fresh pages of the pool: gather just those (on the main
+            # stream, before the next call refills the pool) and bring them back
+            torch.index_select(self.k, 0, self.out_rows, out=self.k_stage)
+            torch.index_select(self.v, 0, self.out_rows, out=self.v_stage)
+            k_res, v_res = self.k_stage, self.v_stage
             out["out_page_table"] = self.h_out_page_table
         else:
-            self.h_k_out.copy_(self.k_out, non_blocking=True)
-            self.h_v_out.copy_(self.v_out, non_blocking=True)
-        self.h_idx.copy_(self.idx, non_blocking=True)
-        self.h_count.copy_(self.count, non_blocking=True)
+            k_res, v_res = self.k_out, self.v_out
+        back = main
+        if overlap_readback:
+            if self._side is None:
+                self._side = torch.cuda.Stream()
+            back = self._side
+            back.wait_stream(main)
+        with torch.cuda.stream(back):
+            self.h_k_out.copy_(k_res, non_blocking=True)
+            self.h_v_out.copy_(v_res, non_blocking=True)
+            if self.paged:
+                self.h_out_page_table.copy_(self.out_page_table, non_blocking=True)
+            self.h_idx.copy_(self.idx, non_blocking=True)
+            self.h_count.copy_(self.count, non_blocking=True)
+            if overlap_readback:
+                self._readback_done = torch.cuda.Event()
+                self._readback_done.record(back)
         return out
+
+    def finish(self) -> None:
+        """Makes the current stream wait for copies back to the host that are still in flight."""
+        if self._readback_done is not None:
+            torch.cuda.current_stream().wait_event(self._readback_done)
+            self._readback_done = None
