@@ -166,7 +166,12 @@ def test_select_negative_and_zero_scores():
 
 
 # ------------------------------------------------------------------ A5
-@pytest.mark.parametrize("n,budget,hkv", [(1, 1, 1), (129, 40, 2), (4099, 4099, 8), (2048, 512, 2)])
+# the last five cases reach the forms of the kernel that move a run of heads per thread group:
+# 2, 4 and all 8 heads of a slot (the batch fills the GPU with fewer units), and head counts that
+# are not powers of two (one unit per slot, the last trip of a unit shorter than the others)
+@pytest.mark.parametrize("n,budget,hkv", [(1, 1, 1), (129, 40, 2), (4099, 4099, 8), (2048, 512, 2),
+                                          (6000, 5000, 8), (12000, 10000, 8), (20000, 19000, 8),
+                                          (700, 650, 6), (700, 300, 3)])
 def test_compact_contiguous(n, budget, hkv):
     rng = np.random.Generator(np.random.PCG64(n + budget))
     k = rng.integers(0, 65535, size=(n, hkv, 128), dtype=np.uint16)
@@ -201,9 +206,14 @@ def test_compact_rejects_in_place_and_bad_index():
     assert ctx().poll() == 0                            # the status word is cleared by the poll
 
 
-def test_compact_paged():
-    wl = gen.Workload("p", 11, 1, 4, 2, 128, 8, gen.POOL_MAX, 3, 0, seq_lens=(100, 37, 260),
-                      budget_frac=0.25, page_size=16)
+@pytest.mark.parametrize("wl", [
+    gen.Workload("p", 11, 1, 4, 2, 128, 8, gen.POOL_MAX, 3, 0, seq_lens=(100, 37, 260),
+                 budget_frac=0.25, page_size=16),
+    # enough slots that a thread group moves four heads of a slot, two groups per slot
+    gen.Workload("p4", 12, 1, 8, 8, 128, 8, gen.POOL_MAX, 3, 0, seq_lens=(9000, 700, 5000, 6300),
+                 budget_frac=0.5, page_size=16),
+], ids=lambda w: w.name)
+def test_compact_paged(wl):
     x = gen.make_layer(wl)
     rng = np.random.Generator(np.random.PCG64(5))
     buds = wl.budgets
