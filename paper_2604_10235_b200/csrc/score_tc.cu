@@ -78,6 +78,12 @@ struct TcParams {
   float* scores;
   float* lse;
   int64_t pool_rows;
+  // K tile in shared memory.  Contiguous cache: two panels of 64 channels, each 128 rows of 128
+  // bytes (8-row groups 1024 bytes apart, second panel 16 KB on).  Paged cache: one copy per page
+  // lays the rows out in 8-token groups of 2 KB, first panel then second (8-row groups of a panel
+  // 2048 bytes apart, second panel 1 KB on), whatever the page size.
+  uint32_t k_sbo16;      // stride between 8-row groups of a panel, in 16-byte units
+  uint32_t k_panel16;    // offset of the second panel, in 16-byte units
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -117,6 +123,14 @@ __device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
       "[%0], [%1, {%3, %4, %5}], [%2], %6;"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy) : "memory");
+}
+// One page of a paged cache: box (64 channels, 8 tokens, 2 panels, page_size / 8 groups, 1 head).
+__device__ __forceinline__ void tma_load_5d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                                 int c3, int c4, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %3, %3, %4, %5}], [%2], %6;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(0), "r"(c3), "r"(c4), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
                                             int c0, int c1, int c2, int c3) {
@@ -392,11 +406,9 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
           // registered before any lane issues a copy
           if (lane == 0) mbar_expect_tx(fb, (uint32_t)__popc(good_mask) * (uint32_t)ps * 256u);
           __syncwarp();
-          if (good) {
-            const uint32_t off = (uint32_t)lane * (uint32_t)ps * 128u;
-            tma_load_3d_hint(dst + off, &k_map, fb, 0, cur.h, page_id * ps, k_policy);
-            tma_load_3d_hint(dst + kPanelBytes + off, &k_map, fb, 64, cur.h, page_id * ps, k_policy);
-          }
+          if (good)      // the page's rows, both panels, in one copy
+            tma_load_5d_hint(dst + (uint32_t)lane * (uint32_t)ps * 256u, &k_map, fb,
+                             page_id * (ps >> 3), cur.h, k_policy);
         }
         if (++stage == P.n_stages) { stage = 0; phase ^= 1; }
       }
@@ -419,7 +431,9 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
       bool need_q = true;
       // descriptor words: low = start address >> 4 | LBO field, high = SBO 1024 B, version 1,
       // 128-byte swizzle
-      const uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+      const uint32_t q_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+      const uint32_t k_hi = P.k_sbo16 | (1u << 14) | (2u << 29);
+      const uint32_t a_hi = PASS == 1 ? q_hi : k_hi, b_hi = PASS == 1 ? k_hi : q_hi;
       const uint32_t q_lo0 = ((smem_u32(q_smem) & 0x3FFFFu) >> 4) | (1u << 16);
       const uint32_t k_lo0 = ((smem_u32(k_smem) & 0x3FFFFu) >> 4) | (1u << 16);
       const uint32_t q_panel16 = q_panel >> 4;
@@ -461,20 +475,20 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
 #pragma unroll
           for (int ks = 0; ks < kHeadDim / 16; ++ks) {
             const uint32_t ql = q_lo + (ks >= 4 ? q_panel16 : 0u) + (uint32_t)(ks & 3) * 2u;
-            const uint32_t kl = k_lo + (ks >= 4 ? (kPanelBytes >> 4) : 0u) + (uint32_t)(ks & 3) * 2u;
+            const uint32_t kl = k_lo + (ks >= 4 ? P.k_panel16 : 0u) + (uint32_t)(ks & 3) * 2u;
             const uint32_t al = PASS == 1 ? ql : kl, bl = PASS == 1 ? kl : ql;
             if (ks == 0) {
               asm volatile(
                   "{\n\t.reg .pred p;\n\t.reg .b64 a, b;\n\tsetp.ne.b32 p, 0, 0;\n\t"
-                  "mov.b64 a, {%1, %3};\n\tmov.b64 b, {%2, %3};\n\t"
+                  "mov.b64 a, {%1, %3};\n\tmov.b64 b, {%2, %5};\n\t"
                   "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %4, p;\n\t}"
-                  ::"r"(d_tmem), "r"(al), "r"(bl), "r"(desc_hi), "r"(idesc) : "memory");
+                  ::"r"(d_tmem), "r"(al), "r"(bl), "r"(a_hi), "r"(idesc), "r"(b_hi) : "memory");
             } else {
               asm volatile(
                   "{\n\t.reg .pred p;\n\t.reg .b64 a, b;\n\tsetp.eq.b32 p, 0, 0;\n\t"
-                  "mov.b64 a, {%1, %3};\n\tmov.b64 b, {%2, %3};\n\t"
+                  "mov.b64 a, {%1, %3};\n\tmov.b64 b, {%2, %5};\n\t"
                   "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %4, p;\n\t}"
-                  ::"r"(d_tmem), "r"(al), "r"(bl), "r"(desc_hi), "r"(idesc) : "memory");
+                  ::"r"(d_tmem), "r"(al), "r"(bl), "r"(a_hi), "r"(idesc), "r"(b_hi) : "memory");
             }
           }
           umma_commit(accf0 + 8u * buf);
@@ -855,16 +869,35 @@ cudaError_t launch_score_tc(const Launch& L, const BatchTable& bt, const Geometr
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { *drv_err = (int)r; return cudaErrorUnknown; }
   }
-  {
+  if (bt.page_size > 0) {
+    // A page (page_size tokens, a multiple of 8, starting at a multiple of 8 rows) as one box: 64
+    // channels x 8 tokens x 2 panels x page_size / 8 groups of one head.  In shared memory that is
+    // page_size / 8 blocks of 2 KB, each the eight rows of the first panel followed by the eight
+    // rows of the second: two copies per page become one (a 16-token page: 4 KB per copy).
+    cuuint64_t dims[5] = {64, 8, 2, (cuuint64_t)(P.pool_rows / 8), (cuuint64_t)g.hkv};
+    cuuint64_t strides[4] = {(cuuint64_t)g.kv_stride_tok * 2, 128, (cuuint64_t)g.kv_stride_tok * 16,
+                             (cuuint64_t)g.kv_stride_head * 2};
+    cuuint32_t box[5] = {64, 8, 2, (cuuint32_t)(bt.page_size / 8), 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUresult r = encode(&k_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(k), dims,
+                        strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { *drv_err = (int)r; return cudaErrorUnknown; }
+    P.k_sbo16 = 2048u >> 4;
+    P.k_panel16 = 1024u >> 4;
+  } else {
     cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)g.hkv, (cuuint64_t)P.pool_rows};
     cuuint64_t strides[2] = {(cuuint64_t)g.kv_stride_head * 2, (cuuint64_t)g.kv_stride_tok * 2};
-    cuuint32_t box[3] = {64, 1, (cuuint32_t)(bt.page_size > 0 ? bt.page_size : kTileKeys)};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)kTileKeys};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = encode(&k_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(k), dims,
                         strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { *drv_err = (int)r; return cudaErrorUnknown; }
+    P.k_sbo16 = 1024u >> 4;
+    P.k_panel16 = kPanelBytes >> 4;
   }
 
   auto pass1 = g.causal ? score_tc_kernel<1, true> : score_tc_kernel<1, false>;
