@@ -62,7 +62,7 @@ def test_scores_tiny_config(mode, tol):
 
 
 @pytest.mark.parametrize("mode,tol", MODES)
-@pytest.mark.parametrize("page", [0, 16, 128])
+@pytest.mark.parametrize("page", [0, 8, 16, 32, 64, 128])      # every supported page size
 def test_scores_ragged_batch(mode, tol, page):
     wl = gen.Workload("ragged", 22, 1, 8, 2, 128, 16, gen.POOL_MAX, 7, 0,
                       seq_lens=(300, 1, 129, 2050, 64), budget_frac=0.1, page_size=page)
