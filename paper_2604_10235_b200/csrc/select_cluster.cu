@@ -34,7 +34,8 @@ constexpr int kDigitBits = 8;
 constexpr int kBins = 1 << kDigitBits;
 constexpr int kCopies = 2;
 constexpr int kMaxCluster = 8;
-constexpr int kCtaItems = 16384;          // items one CTA keeps in shared memory
+constexpr int kCtaItems = 32768;          // items one CTA keeps in shared memory
+constexpr int kStagedItems = 16384;       // up to here the raw scores of the slice are staged there too
 
 struct Shared {
   unsigned hist[2][kCopies][kBins];
@@ -49,6 +50,7 @@ struct ClusterParams {
   int hkv;
   float theta;
   // FUSED only
+  int stage_u;               // the slice's raw scores are staged in shared memory before pooling
   int pool_kind, pool_size;
   float alpha, beta;
   const float* scores;
@@ -369,6 +371,7 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
           if (t0 + k * kThreads < cta_items) keys[padded(t0 + k * kThreads)] = __float_as_uint(b[k]);
       }
       pdl_wait();                                   // the scores are complete from here on
+      if (P.stage_u) {
 #pragma unroll 1
       for (int t0 = threadIdx.x; t0 < span; t0 += 4 * kThreads) {
         float a[4];
@@ -381,8 +384,18 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
         for (int k = 0; k < 4; ++k)
           if (t0 + k * kThreads < span) us[t0 + k * kThreads] = a[k];
       }
+      }
       __syncthreads();
     }
+    // raw score at position t of the staged window (token cta_lo - half + t; zero outside the
+    // sequence): from the staging buffer, or straight from global memory through L1 when the
+    // slice is too long to be staged as well
+    const bool staged = P.stage_u != 0;
+    auto uval = [&](int t) -> float {
+      if (staged) return us[t];
+      const int j = cta_lo - half + t;
+      return (j >= 0 && j < q.n) ? u[j] : 0.0f;
+    };
 #pragma unroll 1
     for (int li = threadIdx.x; li < cta_items; li += kThreads) {
       const int i = cta_lo + li;
@@ -410,14 +423,14 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
       } else {
         pr = __uint_as_float(keys[padded(li)]);       // parked by this very thread
         if (half == 0) {
-          val = us[li];
+          val = uval(li);
         } else if (P.pool_kind == CC_POOL_MAX) {
-          val = us[li + half];
+          val = uval(li + half);
           const int a = max(0, i - half), b = min(q.n - 1, i + half);
-          for (int j = a; j <= b; ++j) val = fmaxf(val, us[j - cta_lo + half]);
+          for (int j = a; j <= b; ++j) val = fmaxf(val, uval(j - cta_lo + half));
         } else {
-          val = us[li];
-          for (int d = 1; d <= 2 * half; ++d) val = __fadd_rn(val, us[li + d]);
+          val = uval(li);
+          for (int d = 1; d <= 2 * half; ++d) val = __fadd_rn(val, uval(li + d));
           val = __fdiv_rn(val, (float)P.pool_size);
         }
       }
@@ -563,18 +576,19 @@ select_cluster_kernel(const __grid_constant__ BatchTable bt, const __grid_consta
   if (c.C > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-size_t cluster_smem_bytes(int per, bool fused, int pool_size) {
+size_t cluster_smem_bytes(int per, bool staged, int pool_size) {
   size_t b = sizeof(Shared);
   b += ((size_t)padded(kThreads * per) + 1) * 4;          // keys
   b += ((size_t)kThreads * per + 15) / 16 * 16;           // flags
-  if (fused) b += ((size_t)kThreads * per + 2 * (pool_size / 2) + 4) * 4;
+  if (staged) b += ((size_t)kThreads * per + 2 * (pool_size / 2) + 4) * 4;
   return (b + 15) / 16 * 16;
 }
 
 }  // namespace
 
 // CTAs per (sequence, head) for the cluster kernel, or 0 when the batch does not fit.
-// A CTA holds up to kCtaItems items (16 per thread); one CTA of 1024 threads fits per SM, and a
+// A CTA holds up to kCtaItems items (32 per thread; the fused form also stages the raw scores of
+// slices of up to 16 per thread and reads them through L1 beyond that); one CTA of 1024 threads fits per SM, and a
 // cluster is placed inside one GPC, so about 96 CTAs run at a time in clusters of eight, 128 in
 // clusters of four, all 148 otherwise.  Wide clusters finish one (sequence, head) sooner, narrow
 // ones let more of them run at once and pay less per exchange (measured: about 6 + 0.6 x width +
@@ -619,7 +633,9 @@ cudaError_t launch_select_cluster(const Launch& L, const BatchTable& bt, const G
   P.idx = idx;
   P.count = count;
   const int per = bt.max_items > 0 ? (bt.max_items + cluster * kThreads - 1) / (cluster * kThreads) : 1;
-  const size_t smem = cluster_smem_bytes(per, fused_input, P.pool_size);
+  // token-level fused form: stage the slice's raw scores while they fit beside keys and flags
+  P.stage_u = fused_input && bt.chunk == 1 && kThreads * per <= kStagedItems ? 1 : 0;
+  const size_t smem = cluster_smem_bytes(per, P.stage_u != 0, P.pool_size);
   const bool chunked = bt.chunk > 1;
   auto kern = fused_input ? (chunked ? select_cluster_kernel<true, true> : select_cluster_kernel<true, false>)
                           : (chunked ? select_cluster_kernel<false, true> : select_cluster_kernel<false, false>);

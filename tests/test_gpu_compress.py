@@ -177,17 +177,21 @@ def test_span_cap_ragged_paged_and_chunked(mode, tol):
     check_layer(wl, gen.make_layer(wl), mode, tol)
 
 
-def test_more_items_than_a_cluster_holds():
-    """A sequence of more than 131072 items: the fused call and cc_topk_select take the
-    single-CTA selection kernel and the stand-alone pooling kernel instead of the cluster kernel."""
-    wl = gen.Workload("long", 36, 1, 2, 1, 128, 8, gen.POOL_MAX, 7, 9000, n=140000)
+@pytest.mark.parametrize("n,pool,k", [(140000, gen.POOL_MAX, 7), (140000, gen.POOL_AVG, 5),
+                                      (270000, gen.POOL_MAX, 7)])
+def test_more_items_than_a_cluster_stages_or_holds(n, pool, k):
+    """140000 items: more than 16 per thread of the widest cluster, so the cluster kernel pools
+    straight from global memory instead of staging the raw scores.  270000 items: more than a
+    cluster holds (262144), so the fused call and cc_topk_select take the single-CTA selection
+    kernel and the stand-alone pooling kernel instead."""
+    wl = gen.Workload("long", 36, 1, 2, 1, 128, 8, pool, k, 9000, n=n)
     x = gen.make_layer(wl)
     check_layer(wl, x, cc.CC_MODE_BF16, 2e-3)
     # selection stage alone on the oracle's fp32 stage values: bit for bit
     from test_gpu_stages import run_select
     rng = np.random.Generator(np.random.PCG64(9))
     u = (np.abs(rng.standard_normal((1, wl.n))) * 1e-3).astype(np.float32)
-    fused = orc.pool_scores(u, orc.POOL_MAX, 7, dtype=np.float32)
+    fused = orc.pool_scores(u, pool, k, dtype=np.float32)
     idx, count = run_select(fused, x.prior, wl.n, wl.budget, wl.force_threshold, 0.5, 16)
     ref = orc.select_tokens(fused[0], x.prior, wl.n, wl.budget, wl.force_threshold, 0.5, 16)
     assert count[0] == len(ref) == wl.budget
