@@ -61,6 +61,16 @@ def test_scores_tiny_config(mode, tol):
     check_against_oracle(wl, gen.make_layer(wl, with_v=False), mode, tol)
 
 
+@pytest.mark.parametrize("w,hq,hkv,page", [(96, 8, 2, 0), (48, 14, 2, 16)])
+def test_scores_three_stage_ring(w, hq, hkv, page):
+    """Row counts of 384 and 336: the shared-memory ring of the tensor-core kernel has three K
+    stages then (four below 313 rows, two above 440), and 40000 keys give every CTA more tiles than
+    the ring has stages, so it wraps."""
+    wl = gen.Workload("ring3", 26, 1, hq, hkv, 128, w, gen.POOL_MAX, 7, 1,
+                      seq_lens=(40000,), budget_frac=0.1, page_size=page)
+    check_against_oracle(wl, gen.make_layer(wl, with_v=False), cc.CC_MODE_BF16, 2e-3)
+
+
 @pytest.mark.parametrize("mode,tol", MODES)
 @pytest.mark.parametrize("page", [0, 8, 16, 32, 64, 128])      # every supported page size
 def test_scores_ragged_batch(mode, tol, page):
