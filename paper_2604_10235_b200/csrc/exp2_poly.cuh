@@ -99,7 +99,12 @@ __device__ __forceinline__ void exp_accumulate(const uint32_t (&v)[32], uint64_t
   for (int i = 0; i < kWidth; i += 4) {
     uint64_t o[2] = {off2, off2};
     if (kPerColumn) {
-      const float4 L = *reinterpret_cast<const float4*>(off_col + i);
+      // off_col is a shared-memory array: a shared-space load with the column offset as an
+      // immediate needs no address arithmetic per load
+      float4 L;
+      asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                   : "=f"(L.x), "=f"(L.y), "=f"(L.z), "=f"(L.w)
+                   : "r"((uint32_t)__cvta_generic_to_shared(off_col) + (uint32_t)(i * 4)));
       o[0] = pack2(L.x, L.y);
       o[1] = pack2(L.z, L.w);
     }

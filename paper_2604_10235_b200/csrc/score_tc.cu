@@ -680,6 +680,8 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
             const int t_row = (sub * 128 + row_in_tile) / g.group;
             if (t_row < g.window) valid_r = min(valid, n_cur - g.window + t_row + 1 - key0);
           }
+          // all 128 keys of the tile count for every row of the warp: no per-chunk range tests
+          const bool full_tile = !kMasked && __shfl_sync(0xffffffffu, valid_r, 0) == kTileKeys;
 #pragma unroll 1
           for (int cc0 = 0; cc0 < kTileKeys; cc0 += 32) {
             if (kMasked) __syncwarp();            // rows of a masked tile skip different chunks
@@ -690,19 +692,27 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
               __syncwarp();
               if (lane == 0) mbar_arrive(empty_bar);
             }
-            if (cc0 >= valid_r) continue;
-            if (cc0 + 32 > valid_r) {
+            if (!full_tile) {
+              if (cc0 >= valid_r) continue;
+              if (cc0 + 32 > valid_r) {
 #pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (cc0 + i >= valid_r) v[i] = 0xc61c4000u;  // -1e4: its exponential underflows to 0
+                for (int i = 0; i < 32; ++i)
+                  if (cc0 + i >= valid_r) v[i] = 0xc61c4000u;  // -1e4: its exponential underflows to 0
+              }
             }
             // The reference of the exponentials only has to be near the row maximum, not equal
-            // to it: it is replaced when a value lies more than 2^64 above it.
+            // to it: it is replaced when a value lies more than 2^64 above it.  The test is a
+            // warp vote where the warp is converged, so that the common case is one uniform branch.
             const float mx = max32(v) * c;
-            if (m_run == -INFINITY || mx > m_run + 64.0f) {
-              if (m_run > -INFINITY) l_run = (l_run + acc_total(acc)) * ex2(m_run - mx);
-              acc[0] = acc[1] = acc[2] = acc[3] = 0ull;
-              m_run = mx;
+            const bool renew = m_run == -INFINITY || mx > m_run + 64.0f;
+            // (the rows of a masked tile skip different chunks, so its lanes are not converged
+            // here and must not vote; everywhere else the warp takes this path as one)
+            if (kMasked ? renew : __any_sync(0xffffffffu, renew)) {
+              if (renew) {
+                if (m_run > -INFINITY) l_run = (l_run + acc_total(acc)) * ex2(m_run - mx);
+                acc[0] = acc[1] = acc[2] = acc[3] = 0ull;
+                m_run = mx;
+              }
             }
             exp_accumulate<false, 32>(v, c2, pack2(-m_run, -m_run), nullptr, acc);
           }
