@@ -90,21 +90,22 @@ __device__ __forceinline__ uint64_t ex2_pair_fma(uint64_t x) {
 constexpr int kPolyEvery = CC_POLY_EVERY;        // one pair in this many takes the polynomial path
 
 // acc += 2^(v * c + off) over the first kWidth of 32 values; off is one pair for all of them or
-// read per value from shared memory.  Of every kPolyEvery pairs one goes to the FMA pipe, the
+// read per value from shared memory (off_col: shared-space address of the first value's offset).
+// Of every kPolyEvery pairs one goes to the FMA pipe, the
 // others to the special-function unit.
 template <bool kPerColumn, int kWidth>
 __device__ __forceinline__ void exp_accumulate(const uint32_t (&v)[32], uint64_t c2, uint64_t off2,
-                                               const float* off_col, uint64_t (&acc)[4]) {
+                                               uint32_t off_col, uint64_t (&acc)[4]) {
 #pragma unroll
   for (int i = 0; i < kWidth; i += 4) {
     uint64_t o[2] = {off2, off2};
     if (kPerColumn) {
-      // off_col is a shared-memory array: a shared-space load with the column offset as an
-      // immediate needs no address arithmetic per load
+      // off_col is the shared-space address of the offsets: a shared-space load at a constant
+      // distance from it needs no address arithmetic per load
       float4 L;
       asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
                    : "=f"(L.x), "=f"(L.y), "=f"(L.z), "=f"(L.w)
-                   : "r"((uint32_t)__cvta_generic_to_shared(off_col) + (uint32_t)(i * 4)));
+                   : "r"(off_col + (uint32_t)(i * 4)));
       o[0] = pack2(L.x, L.y);
       o[1] = pack2(L.z, L.w);
     }

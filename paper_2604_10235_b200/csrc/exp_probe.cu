@@ -65,7 +65,7 @@ exp_probe_kernel(long long* out, int iters, float c, float off) {
     } else {
       off2 = add2(off2, pack2(-1.0e-4f, -1.0e-4f));     // new arguments every round
     }
-    exp_accumulate<false, 32>(v, c2, off2, nullptr, acc);
+    exp_accumulate<false, 32>(v, c2, off2, 0u, acc);
   }
   const long long t1 = clock64();
   const float total = acc_total(acc);

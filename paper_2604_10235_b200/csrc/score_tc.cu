@@ -714,7 +714,7 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
                 m_run = mx;
               }
             }
-            exp_accumulate<false, 32>(v, c2, pack2(-m_run, -m_run), nullptr, acc);
+            exp_accumulate<false, 32>(v, c2, pack2(-m_run, -m_run), 0u, acc);
           }
           };
           if (CAUSAL && masked_tile) drain(std::true_type{}); else drain(std::false_type{});
@@ -730,7 +730,7 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
           // thread = key (key0 + row_in_tile); columns = the query rows of this chunk
           const int c0 = sub * P.sub_cols;
           const int nc = min(P.sub_cols, P.rows_pad - c0);        // multiple of 16
-          const float* nl = misc->neg_lc + c0;
+          const uint32_t nl = smem_u32(misc->neg_lc + c0);         // -L_r of the item's columns
           // causal window: key j is seen by the rows t >= j - (n - w), i.e. by the columns
           // from G * (j - n + w) on; the columns before it contribute nothing
           const bool masked_tile = CAUSAL && key0 + kTileKeys > n_cur - g.window + 1;
@@ -752,8 +752,8 @@ score_tc_kernel(const __grid_constant__ BatchTable bt, const __grid_constant__ G
               __syncwarp();
               if (lane == 0) mbar_arrive(empty_bar);
             }
-            if (cc0 + 32 <= nc) exp_accumulate<true, 32>(v, c2, 0ull, nl + cc0, acc);
-            else                exp_accumulate<true, 16>(v, c2, 0ull, nl + cc0, acc);
+            if (cc0 + 32 <= nc) exp_accumulate<true, 32>(v, c2, 0ull, nl + 4u * (uint32_t)cc0, acc);
+            else                exp_accumulate<true, 16>(v, c2, 0ull, nl + 4u * (uint32_t)cc0, acc);
           }
           };
           if (CAUSAL && masked_tile) drain(std::true_type{}); else drain(std::false_type{});
